@@ -1,0 +1,178 @@
+/*
+ * quoka.h - C ABI of the B200 (sm_100a) implementation of QuoKA's per-chunk
+ * sparse prefill attention ("QuoKA: Query-oriented KV selection for efficient
+ * LLM prefill", Algorithm 1 and Algorithm 2).
+ *
+ * One call sequence handles ONE attention layer and ONE prefill chunk of every
+ * sequence in a batch:
+ *
+ *   quoka_select_queries   Alg. 1 "Query Sub-selection" + normalisation + GQA pre-aggregation
+ *   quoka_score_keys       Alg. 1  S = Qbar K^T on normalised keys,  S^ = max over queries
+ *   quoka_select_keys      Alg. 1  I = topk(S^, B_SA)
+ *   quoka_sparse_attn      Alg. 2  Attention(Q_i, [K^ | K_i], [V^ | V_i])   (Eq. 1, Eq. 2)
+ *   quoka_prefill_chunk    all four, back to back on one stream
+ *   quoka_dense_chunk_attn Eq. 2 without selection (the speed-up denominator)
+ *
+ * Symbols: b batch, n_Q query heads, n_KV KV heads, G = n_Q / n_KV, d head_dim,
+ * T_s cached length of sequence s (K_<i), C = B_CP chunk length, N = min(N_Q, C)
+ * retained queries, B_s = key budget of sequence s.
+ *
+ * Pointers.  Unless a parameter is marked HOST, every data pointer is a DEVICE
+ * pointer into memory the caller allocated; the library allocates nothing, keeps
+ * no state between calls (except the entry point marked otherwise) and only
+ * writes the outputs and the workspace.  `stream` is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  Calls are asynchronous: they
+ * enqueue work on `stream` and return.
+ *
+ * Cache layout.  The caller has ALREADY written the chunk's own K_i, V_i at rows
+ * [T_s, T_s + C) of the cache (Alg. 2 appends after attention; appending before
+ * is equivalent because selection only reads rows < T_s).  Contiguous cache:
+ * element (s, h, t, x) at  s*kv_stride_b + h*kv_stride_h + t*kv_stride_t + x.
+ * Paged cache (page_size == 64): logical row t of sequence s lives in page
+ * p = block_table[s*max_pages_per_seq + t/64] at
+ * p*kv_stride_b + h*kv_stride_h + (t%64)*kv_stride_t + x.   Strides are in
+ * elements; head_dim is contiguous.  All base pointers 16-byte aligned, all
+ * strides multiples of 8 elements.
+ *
+ * Errors.  Every call validates its arguments on the host before launching
+ * anything and returns a status; nothing is launched on error.  Problems only
+ * the device can see (a bounded wait that ran out) are recorded in a status word
+ * inside the workspace: read it with quoka_last_device_status.  No entry point
+ * throws, traps or blocks.
+ *
+ * Determinism.  The same inputs give bit-identical outputs from run to run.
+ */
+#ifndef QUOKA_H_
+#define QUOKA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QUOKA_OK = 0,
+  QUOKA_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, n_Q % n_KV != 0, misaligned stride */
+  QUOKA_ERR_UNSUPPORTED = 2,  /* head_dim not in {64,128}, page_size not in {0,64}, chunk_len > 8192 with selection */
+  QUOKA_ERR_WORKSPACE = 3,    /* workspace pointer null / misaligned / smaller than quoka_workspace_size */
+  QUOKA_ERR_CUDA = 4,         /* a CUDA runtime or driver call failed (launch, tensor-map encode) */
+  QUOKA_ERR_TIMEOUT = 5       /* device status word: a bounded wait inside a kernel ran out */
+} quoka_status;
+
+typedef enum { QUOKA_BF16 = 0, QUOKA_F32 = 1 } quoka_dtype;
+
+/* Which kernels serve the contraction steps (scoring, attention). */
+typedef enum {
+  QUOKA_IMPL_AUTO = 0,   /* tcgen05 tensor-core kernels for bf16, scalar kernels for f32 */
+  QUOKA_IMPL_SIMT = 1,   /* scalar fp32 kernels (any dtype); the on-device cross-check */
+  QUOKA_IMPL_TENSOR = 2  /* tcgen05 kernels; QUOKA_ERR_UNSUPPORTED if dtype is f32 */
+} quoka_impl;
+
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim;
+  int32_t chunk_len;     /* C = B_CP                                                          */
+  int32_t n_retain;      /* N_Q; >= chunk_len means no query sub-selection (Alg. 1, the `if`)  */
+  int32_t kv_budget;     /* B_SA in keys, B_s = min(B_SA, T_s); <= 0 selects budget_frac       */
+  float budget_frac;     /* B_s = floor(budget_frac * T_s + 0.5), evaluated in double          */
+  int32_t dtype;         /* quoka_dtype of q, k_cache, v_cache, qbar, out                      */
+  int32_t impl;          /* quoka_impl                                                         */
+  float softmax_scale;   /* 0 selects 1/sqrt(head_dim) (Eq. 1)                                 */
+  int32_t max_ctx_len;   /* HOST upper bound on every T_s: sizes grids, buffers and workspace  */
+  const int32_t* ctx_len;      /* DEVICE [batch]: T_s; rows [0,T_s) are the selectable cache    */
+  /* q and out: element (s, h, r, x) at s*stride_b + h*stride_h + r*stride_t + x               */
+  int64_t q_stride_b, q_stride_h, q_stride_t;
+  int64_t o_stride_b, o_stride_h, o_stride_t;
+  /* KV cache, see "Cache layout" above                                                        */
+  int32_t page_size;           /* 0 = contiguous, 64 = paged                                    */
+  int32_t max_pages_per_seq;
+  const int32_t* block_table;  /* DEVICE [batch][max_pages_per_seq], NULL when contiguous       */
+  int64_t kv_stride_b, kv_stride_h, kv_stride_t;   /* kv_stride_b is the page stride when paged */
+  int64_t kv_rows;             /* rows allocated per (sequence, head) when contiguous (>= T_s+C);
+                                  number of pages in the pool when paged                        */
+} quoka_params;
+
+/* Row pitch of k_idx: the largest B_s any sequence can have, from max_ctx_len. */
+quoka_status quoka_kv_budget_cap(const quoka_params* p, int32_t* cap);
+
+/* Bytes of workspace that every call below accepts (256-byte aligned pointer).
+ * The first 256 bytes hold the device status word, which the caller sets to zero
+ * once after allocating; the rest is scratch whose contents mean nothing between
+ * calls.  Two calls that share a workspace must not overlap on the GPU. */
+quoka_status quoka_workspace_size(const quoka_params* p, size_t* bytes);
+
+/* Alg. 1, "Query Sub-selection", then the normalisation and the mean over the G
+ * heads of each KV group.  Per query head: M = mean over the chunk of the raw
+ * queries; c_r = CosSim(q_r, M); if C > N_Q keep the N_Q rows of LOWEST c_r,
+ * most dissimilar first, equal values earlier position first, else keep all rows
+ * in order.  Then Qbar[kv][j] = (1/G) sum_g  q^_{kvG+g, pi_g(j)}  with
+ * q^ = q / max(|q|, 1e-12), accumulated in fp32 and rounded once to `dtype`.
+ *   q      in  [b][n_Q][C][d] by strides
+ *   q_idx  out [b][n_Q][N] int32, ordered by rank
+ *   qbar   out [b][n_KV][N][d] dense, `dtype` */
+quoka_status quoka_select_queries(const quoka_params* p, const void* q, int32_t* q_idx, void* qbar,
+                                  void* ws, size_t ws_bytes, void* stream);
+
+/* Alg. 1, scoring and max over the query axis: for every cached row t < T_s,
+ * scores[s][kv][t] = max_j (Qbar[s][kv][j] . k_t) / max(|k_t|, 1e-12).  The
+ * N x T score matrix is never written to memory.
+ *   scores out [b][n_KV][max_ctx_len] fp32; entries t >= T_s are not written */
+quoka_status quoka_score_keys(const quoka_params* p, const void* qbar, const void* k_cache, float* scores,
+                              void* ws, size_t ws_bytes, void* stream);
+
+/* Alg. 1, I = topk(S^, B_SA) per (sequence, KV head): the B_s rows with the
+ * largest score; among equal scores at the threshold the lower row wins; the
+ * list is written ascending by row.  T_s <= B_s gives 0..T_s-1.
+ *   k_idx out [b][n_KV][cap] int32 (cap from quoka_kv_budget_cap), entries >= B_s set to -1
+ *   k_cnt out [b] int32 = B_s */
+quoka_status quoka_select_keys(const quoka_params* p, const float* scores, int32_t* k_idx, int32_t* k_cnt,
+                               void* ws, size_t ws_bytes, void* stream);
+
+/* Alg. 2, the attention line, with Eq. 1/Eq. 2 semantics: row r of query head h
+ * attends rows k_idx[s][h/G][0..k_cnt[s]) of the ORIGINAL cache plus the chunk's
+ * own rows T_s..T_s+r (causal, diagonal included); softmax in fp32.  The rows are
+ * gathered inside the kernel; no compacted copy of K or V is made.
+ *   out [b][n_Q][C][d] by strides, `dtype`;  lse [b][n_Q][C] fp32 natural-log-sum-exp of
+ *   the scaled logits, may be NULL */
+quoka_status quoka_sparse_attn(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse,
+                               void* ws, size_t ws_bytes, void* stream);
+
+/* Eq. 2: the chunk attends all T_s cached rows and its own rows causally. */
+quoka_status quoka_dense_chunk_attn(const quoka_params* p, const void* q, const void* k_cache,
+                                    const void* v_cache, void* out, float* lse,
+                                    void* ws, size_t ws_bytes, void* stream);
+
+/* Alg. 2, loop body: the four steps above on `stream` with the intermediates in
+ * the workspace.  k_idx_out ([b][n_KV][cap]) and k_cnt_out ([b]) may be NULL; when
+ * given they receive the selection that was used. */
+quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                                 void* out, int32_t* k_idx_out, int32_t* k_cnt_out,
+                                 void* ws, size_t ws_bytes, void* stream);
+
+/* The same loop body for a caller whose chunk lives in HOST memory (pinned for
+ * the copies to be asynchronous): copies q_host -> q_dev, the chunk's K_i, V_i
+ * ([b][n_KV][C][d] dense, HOST) into rows [T_s, T_s+C) of the contiguous device
+ * cache, runs quoka_prefill_chunk, and copies out_dev -> out_host
+ * ([b][n_Q][C][d] dense), all on `stream`.  ctx_len_host is a HOST copy of T_s.
+ * Paged caches are not supported here (QUOKA_ERR_UNSUPPORTED).  q_dev / out_dev
+ * must be dense [b][n_Q][C][d] and p's q/o strides must describe them. */
+quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_len_host,
+                                      const void* q_host, const void* k_new_host, const void* v_new_host,
+                                      void* out_host, void* q_dev, void* k_cache, void* v_cache, void* out_dev,
+                                      void* ws, size_t ws_bytes, void* stream);
+
+/* Copies the device status word of `ws` to the host (synchronises `stream`) and
+ * clears it.  *status_out is a quoka_status. */
+quoka_status quoka_last_device_status(void* ws, void* stream, int32_t* status_out);
+
+const char* quoka_status_string(quoka_status s);
+
+/* Number of kernels this library has launched in this process (all entry points). */
+int64_t quoka_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QUOKA_H_ */

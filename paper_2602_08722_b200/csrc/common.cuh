@@ -1,0 +1,141 @@
+// Shared device-side definitions for the QuoKA kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "quoka.h"
+
+namespace quoka {
+
+constexpr float kNormEps = 1e-12f;
+constexpr int kPage = 64;
+
+// Device copy of the launch-invariant part of quoka_params.
+struct DevParams {
+  int batch, n_q, n_kv, group, d;
+  int chunk;        // C
+  int n_sel;        // N = min(N_Q, C)
+  int n_retain;     // N_Q as given
+  int kv_budget;    // B_SA or <= 0
+  float budget_frac;
+  float scale;      // softmax scale
+  int max_ctx;
+  int budget_cap;   // row pitch of k_idx
+  const int32_t* ctx_len;
+  int64_t q_sb, q_sh, q_st;
+  int64_t o_sb, o_sh, o_st;
+  int page_size, max_pages;
+  const int32_t* block_table;
+  int64_t kv_sb, kv_sh, kv_st;
+  int32_t* status;  // device status word
+};
+
+// B_s of one sequence: min(B_SA, T) or floor(frac*T + 0.5) in double.
+__host__ __device__ inline int key_budget(int T, int kv_budget, float frac) {
+  if (kv_budget > 0) return kv_budget < T ? kv_budget : T;
+  int B = (int)floor((double)frac * (double)T + 0.5);
+  if (B < 0) B = 0;
+  return B < T ? B : T;
+}
+
+// Element offset of row t of (sequence s, KV head h) in a contiguous or paged cache.
+__device__ __forceinline__ int64_t kv_row_offset(const DevParams& P, int s, int h, int t) {
+  if (P.page_size == 0) return (int64_t)s * P.kv_sb + (int64_t)h * P.kv_sh + (int64_t)t * P.kv_st;
+  const int page = __ldg(P.block_table + (int64_t)s * P.max_pages + (t >> 6));
+  return (int64_t)page * P.kv_sb + (int64_t)h * P.kv_sh + (int64_t)(t & (kPage - 1)) * P.kv_st;
+}
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Load NE consecutive elements (NE*sizeof(T) is 8, 16 or 32 bytes, pointer aligned to min(16, that)) as floats.
+template <typename T, int NE>
+__device__ __forceinline__ void load_vec(const T* __restrict__ p, float (&out)[NE]) {
+  if constexpr (sizeof(T) == 4) {
+    if constexpr (NE % 4 == 0) {
+#pragma unroll
+      for (int i = 0; i < NE / 4; ++i) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p) + i);
+        out[4 * i + 0] = v.x; out[4 * i + 1] = v.y; out[4 * i + 2] = v.z; out[4 * i + 3] = v.w;
+      }
+    } else {
+      static_assert(NE % 2 == 0, "NE");
+#pragma unroll
+      for (int i = 0; i < NE / 2; ++i) {
+        const float2 v = __ldg(reinterpret_cast<const float2*>(p) + i);
+        out[2 * i] = v.x; out[2 * i + 1] = v.y;
+      }
+    }
+  } else {
+    if constexpr (NE % 8 == 0) {
+#pragma unroll
+      for (int i = 0; i < NE / 8; ++i) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p) + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          out[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+          out[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+        }
+      }
+    } else if constexpr (NE % 4 == 0) {
+#pragma unroll
+      for (int i = 0; i < NE / 4; ++i) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(p) + i);
+        out[4 * i + 0] = __uint_as_float(v.x << 16); out[4 * i + 1] = __uint_as_float(v.x & 0xFFFF0000u);
+        out[4 * i + 2] = __uint_as_float(v.y << 16); out[4 * i + 3] = __uint_as_float(v.y & 0xFFFF0000u);
+      }
+    } else {
+      static_assert(NE % 2 == 0, "NE");
+#pragma unroll
+      for (int i = 0; i < NE / 2; ++i) {
+        const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(p) + i);
+        out[2 * i] = __uint_as_float(v << 16); out[2 * i + 1] = __uint_as_float(v & 0xFFFF0000u);
+      }
+    }
+  }
+}
+
+template <typename T, int NE>
+__device__ __forceinline__ void store_vec(T* __restrict__ p, const float (&v)[NE]) {
+#pragma unroll
+  for (int i = 0; i < NE; ++i) p[i] = from_f32<T>(v[i]);
+}
+
+// Monotone map float -> uint32 (ascending); -0 and +0 map to the same code.
+__device__ __forceinline__ uint32_t float_order_key(float f) {
+  uint32_t b = __float_as_uint(f);
+  if ((b << 1) == 0) b = 0;
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+  return x;
+}
+
+// ---- launch functions implemented in the .cu files (host side) -------------------------------
+struct Launch {
+  cudaStream_t stream;
+};
+
+cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st);
+cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, const int32_t* q_idx, void* qbar,
+                                     cudaStream_t st);
+cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,
+                                   cudaStream_t st);
+cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt,
+                               cudaStream_t st);
+cudaError_t launch_attn_simt(const DevParams& P, int dtype, const void* q, const void* k, const void* v,
+                             const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st);
+
+void count_launch(int n = 1);
+
+}  // namespace quoka

@@ -1,0 +1,299 @@
+// Host side of the C ABI: argument validation, workspace carving, launch sequencing.
+// Nothing here allocates device memory or synchronises (except quoka_last_device_status).
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+
+#include "common.cuh"
+#include "tensor_kernels.cuh"
+
+namespace quoka {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Workspace {
+  int32_t* status;
+  int32_t* q_idx;
+  void* qbar;
+  float* scores;
+  int32_t* k_idx;
+  int32_t* k_cnt;
+  size_t total;
+};
+
+static int budget_cap_of(const quoka_params* p) {
+  int cap = key_budget(p->max_ctx_len, p->kv_budget, p->budget_frac);
+  return cap < 1 ? 1 : cap;
+}
+
+static Workspace carve(const quoka_params* p, void* ws) {
+  Workspace w{};
+  const size_t es = p->dtype == QUOKA_BF16 ? 2 : 4;
+  const int N = p->n_retain < p->chunk_len ? p->n_retain : p->chunk_len;
+  const int cap = budget_cap_of(p);
+  char* base = static_cast<char*>(ws);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    char* r = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return r;
+  };
+  w.status = reinterpret_cast<int32_t*>(take(256));
+  w.q_idx = reinterpret_cast<int32_t*>(take((size_t)p->batch * p->n_q_heads * N * 4));
+  w.qbar = take((size_t)p->batch * p->n_kv_heads * N * p->head_dim * es);
+  w.scores = reinterpret_cast<float*>(take((size_t)p->batch * p->n_kv_heads * (size_t)(p->max_ctx_len > 0 ? p->max_ctx_len : 1) * 4));
+  w.k_idx = reinterpret_cast<int32_t*>(take((size_t)p->batch * p->n_kv_heads * cap * 4));
+  w.k_cnt = reinterpret_cast<int32_t*>(take((size_t)p->batch * 4));
+  w.total = off;
+  return w;
+}
+
+static quoka_status validate(const quoka_params* p) {
+  if (!p) return QUOKA_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->chunk_len <= 0 || p->n_retain <= 0)
+    return QUOKA_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads != 0) return QUOKA_ERR_INVALID_ARG;
+  if (p->max_ctx_len < 0 || !p->ctx_len) return QUOKA_ERR_INVALID_ARG;
+  if (p->kv_budget <= 0 && !(p->budget_frac >= 0.f && p->budget_frac <= 1.f)) return QUOKA_ERR_INVALID_ARG;
+  if (p->dtype != QUOKA_BF16 && p->dtype != QUOKA_F32) return QUOKA_ERR_INVALID_ARG;
+  if (p->impl < QUOKA_IMPL_AUTO || p->impl > QUOKA_IMPL_TENSOR) return QUOKA_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return QUOKA_ERR_UNSUPPORTED;
+  if (p->page_size != 0 && p->page_size != kPage) return QUOKA_ERR_UNSUPPORTED;
+  if (p->page_size == kPage && (!p->block_table || p->max_pages_per_seq <= 0)) return QUOKA_ERR_INVALID_ARG;
+  if (p->page_size == kPage && (int64_t)p->max_pages_per_seq * kPage < (int64_t)p->max_ctx_len + p->chunk_len)
+    return QUOKA_ERR_INVALID_ARG;
+  if (p->page_size == 0 && p->kv_rows < (int64_t)p->max_ctx_len + p->chunk_len) return QUOKA_ERR_INVALID_ARG;
+  if (p->chunk_len > p->n_retain && p->chunk_len > 8192) return QUOKA_ERR_UNSUPPORTED;
+  if (p->impl == QUOKA_IMPL_TENSOR && p->dtype != QUOKA_BF16) return QUOKA_ERR_UNSUPPORTED;
+  const int64_t strides[] = {p->q_stride_b, p->q_stride_h, p->q_stride_t, p->o_stride_b, p->o_stride_h,
+                             p->o_stride_t, p->kv_stride_b, p->kv_stride_h, p->kv_stride_t};
+  for (int64_t s : strides)
+    if (s < 0 || (s % 8) != 0) return QUOKA_ERR_INVALID_ARG;
+  if (p->q_stride_t < p->head_dim || p->o_stride_t < p->head_dim || p->kv_stride_t < p->head_dim)
+    return QUOKA_ERR_INVALID_ARG;
+  return QUOKA_OK;
+}
+
+static bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }
+
+static quoka_status check_ws(const quoka_params* p, void* ws, size_t ws_bytes) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0) return QUOKA_ERR_WORKSPACE;
+  if (ws_bytes < carve(p, nullptr).total) return QUOKA_ERR_WORKSPACE;
+  return QUOKA_OK;
+}
+
+static DevParams make_dev(const quoka_params* p, void* ws) {
+  DevParams P{};
+  P.batch = p->batch; P.n_q = p->n_q_heads; P.n_kv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
+  P.d = p->head_dim; P.chunk = p->chunk_len; P.n_retain = p->n_retain;
+  P.n_sel = p->n_retain < p->chunk_len ? p->n_retain : p->chunk_len;
+  P.kv_budget = p->kv_budget; P.budget_frac = p->budget_frac;
+  P.scale = p->softmax_scale != 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  P.max_ctx = p->max_ctx_len; P.budget_cap = budget_cap_of(p);
+  P.ctx_len = p->ctx_len;
+  P.q_sb = p->q_stride_b; P.q_sh = p->q_stride_h; P.q_st = p->q_stride_t;
+  P.o_sb = p->o_stride_b; P.o_sh = p->o_stride_h; P.o_st = p->o_stride_t;
+  P.page_size = p->page_size; P.max_pages = p->max_pages_per_seq; P.block_table = p->block_table;
+  P.kv_sb = p->kv_stride_b; P.kv_sh = p->kv_stride_h; P.kv_st = p->kv_stride_t;
+  P.status = static_cast<int32_t*>(ws);
+  return P;
+}
+
+static bool use_tensor(const quoka_params* p) {
+  if (p->impl == QUOKA_IMPL_SIMT) return false;
+  if (p->dtype != QUOKA_BF16) return false;
+  return true;
+}
+
+#define QUOKA_TRY_CUDA(expr)                          \
+  do {                                                \
+    cudaError_t e_ = (expr);                          \
+    if (e_ != cudaSuccess) return QUOKA_ERR_CUDA;     \
+  } while (0)
+
+static quoka_status run_select_queries(const quoka_params* p, const DevParams& P, const void* q, int32_t* q_idx,
+                                       void* qbar, cudaStream_t st) {
+  QUOKA_TRY_CUDA(launch_rank_queries(P, p->dtype, q, q_idx, st));
+  QUOKA_TRY_CUDA(launch_aggregate_queries(P, p->dtype, q, q_idx, qbar, st));
+  return QUOKA_OK;
+}
+
+static quoka_status run_score_keys(const quoka_params* p, const DevParams& P, const void* qbar, const void* k,
+                                   float* scores, cudaStream_t st) {
+  if (p->max_ctx_len == 0) return QUOKA_OK;
+  if (use_tensor(p) && score_keys_tc_supported(p)) return launch_score_keys_tc(p, P, qbar, k, scores, st);
+  if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;
+  QUOKA_TRY_CUDA(launch_score_keys_simt(P, p->dtype, qbar, k, scores, st));
+  return QUOKA_OK;
+}
+
+static quoka_status run_attn(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
+                             const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st) {
+  if (use_tensor(p) && attn_tc_supported(p)) return launch_attn_tc(p, P, q, k, v, k_idx, k_cnt, out, lse, st);
+  if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;
+  QUOKA_TRY_CUDA(launch_attn_simt(P, p->dtype, q, k, v, k_idx, k_cnt, out, lse, st));
+  return QUOKA_OK;
+}
+
+}  // namespace quoka
+
+using namespace quoka;
+
+extern "C" {
+
+quoka_status quoka_kv_budget_cap(const quoka_params* p, int32_t* cap) {
+  if (!p || !cap) return QUOKA_ERR_INVALID_ARG;
+  *cap = budget_cap_of(p);
+  return QUOKA_OK;
+}
+
+quoka_status quoka_workspace_size(const quoka_params* p, size_t* bytes) {
+  if (!bytes) return QUOKA_ERR_INVALID_ARG;
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  *bytes = carve(p, nullptr).total;
+  return QUOKA_OK;
+}
+
+quoka_status quoka_select_queries(const quoka_params* p, const void* q, int32_t* q_idx, void* qbar, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!q || !q_idx || !qbar || !aligned16(q) || !aligned16(qbar)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  return run_select_queries(p, make_dev(p, ws), q, q_idx, qbar, static_cast<cudaStream_t>(stream));
+}
+
+quoka_status quoka_score_keys(const quoka_params* p, const void* qbar, const void* k_cache, float* scores, void* ws,
+                              size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!qbar || !k_cache || !scores || !aligned16(qbar) || !aligned16(k_cache)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  return run_score_keys(p, make_dev(p, ws), qbar, k_cache, scores, static_cast<cudaStream_t>(stream));
+}
+
+quoka_status quoka_select_keys(const quoka_params* p, const float* scores, int32_t* k_idx, int32_t* k_cnt, void* ws,
+                               size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!scores || !k_idx || !k_cnt) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  DevParams P = make_dev(p, ws);
+  QUOKA_TRY_CUDA(launch_select_keys(P, scores, k_idx, k_cnt, static_cast<cudaStream_t>(stream)));
+  return QUOKA_OK;
+}
+
+quoka_status quoka_sparse_attn(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, void* ws,
+                               size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!q || !k_cache || !v_cache || !k_idx || !k_cnt || !out) return QUOKA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  return run_attn(p, make_dev(p, ws), q, k_cache, v_cache, k_idx, k_cnt, out, lse,
+                  static_cast<cudaStream_t>(stream));
+}
+
+quoka_status quoka_dense_chunk_attn(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                                    void* out, float* lse, void* ws, size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!q || !k_cache || !v_cache || !out) return QUOKA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  return run_attn(p, make_dev(p, ws), q, k_cache, v_cache, nullptr, nullptr, out, lse,
+                  static_cast<cudaStream_t>(stream));
+}
+
+quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                                 void* out, int32_t* k_idx_out, int32_t* k_cnt_out, void* ws, size_t ws_bytes,
+                                 void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!q || !k_cache || !v_cache || !out) return QUOKA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  DevParams P = make_dev(p, ws);
+  Workspace w = carve(p, ws);
+  int32_t* k_idx = k_idx_out ? k_idx_out : w.k_idx;
+  int32_t* k_cnt = k_cnt_out ? k_cnt_out : w.k_cnt;
+  if (p->max_ctx_len > 0) {
+    if ((st = run_select_queries(p, P, q, w.q_idx, w.qbar, cs)) != QUOKA_OK) return st;
+    if ((st = run_score_keys(p, P, w.qbar, k_cache, w.scores, cs)) != QUOKA_OK) return st;
+  }
+  // with an empty cache the selection kernel only writes k_cnt = 0 and the -1 padding
+  QUOKA_TRY_CUDA(launch_select_keys(P, w.scores, k_idx, k_cnt, cs));
+  return run_attn(p, P, q, k_cache, v_cache, k_idx, k_cnt, out, nullptr, cs);
+}
+
+quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_len_host, const void* q_host,
+                                      const void* k_new_host, const void* v_new_host, void* out_host, void* q_dev,
+                                      void* k_cache, void* v_cache, void* out_dev, void* ws, size_t ws_bytes,
+                                      void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (p->page_size != 0) return QUOKA_ERR_UNSUPPORTED;
+  if (!ctx_len_host || !q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_cache || !v_cache ||
+      !out_dev)
+    return QUOKA_ERR_INVALID_ARG;
+  const size_t es = p->dtype == QUOKA_BF16 ? 2 : 4;
+  const int64_t C = p->chunk_len, d = p->head_dim;
+  if (p->q_stride_t != d || p->q_stride_h != C * d || p->q_stride_b != (int64_t)p->n_q_heads * C * d ||
+      p->o_stride_t != d || p->o_stride_h != C * d || p->o_stride_b != (int64_t)p->n_q_heads * C * d ||
+      p->kv_stride_t != d)
+    return QUOKA_ERR_INVALID_ARG;
+  for (int s = 0; s < p->batch; ++s)
+    if (ctx_len_host[s] < 0 || ctx_len_host[s] > p->max_ctx_len) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const size_t q_bytes = (size_t)p->batch * p->n_q_heads * C * d * es;
+  QUOKA_TRY_CUDA(cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, cs));
+  for (int s = 0; s < p->batch; ++s) {
+    const size_t dst_off = ((size_t)s * p->kv_stride_b + (size_t)ctx_len_host[s] * p->kv_stride_t) * es;
+    const size_t src_off = (size_t)s * p->n_kv_heads * C * d * es;
+    QUOKA_TRY_CUDA(cudaMemcpy2DAsync(static_cast<char*>(k_cache) + dst_off, (size_t)p->kv_stride_h * es,
+                                     static_cast<const char*>(k_new_host) + src_off, (size_t)C * d * es,
+                                     (size_t)C * d * es, p->n_kv_heads, cudaMemcpyHostToDevice, cs));
+    QUOKA_TRY_CUDA(cudaMemcpy2DAsync(static_cast<char*>(v_cache) + dst_off, (size_t)p->kv_stride_h * es,
+                                     static_cast<const char*>(v_new_host) + src_off, (size_t)C * d * es,
+                                     (size_t)C * d * es, p->n_kv_heads, cudaMemcpyHostToDevice, cs));
+  }
+  st = quoka_prefill_chunk(p, q_dev, k_cache, v_cache, out_dev, nullptr, nullptr, ws, ws_bytes, stream);
+  if (st != QUOKA_OK) return st;
+  QUOKA_TRY_CUDA(cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, cs));
+  return QUOKA_OK;
+}
+
+quoka_status quoka_last_device_status(void* ws, void* stream, int32_t* status_out) {
+  if (!ws || !status_out) return QUOKA_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  int32_t h = 0;
+  QUOKA_TRY_CUDA(cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, cs));
+  QUOKA_TRY_CUDA(cudaStreamSynchronize(cs));
+  QUOKA_TRY_CUDA(cudaMemsetAsync(ws, 0, sizeof(int32_t), cs));
+  *status_out = h;
+  return QUOKA_OK;
+}
+
+const char* quoka_status_string(quoka_status s) {
+  switch (s) {
+    case QUOKA_OK: return "ok";
+    case QUOKA_ERR_INVALID_ARG: return "invalid argument";
+    case QUOKA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case QUOKA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case QUOKA_ERR_CUDA: return "CUDA call failed";
+    case QUOKA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int64_t quoka_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,17 @@
+// Host-side entry points of the tcgen05 (5th-generation tensor core) kernels.
+#pragma once
+
+#include "common.cuh"
+
+namespace quoka {
+
+// Whether the tensor-core kernel covers this configuration (bf16, supported N / head_dim / layout).
+bool score_keys_tc_supported(const quoka_params* p);
+quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, const void* qbar, const void* k,
+                                  float* scores, cudaStream_t st);
+
+bool attn_tc_supported(const quoka_params* p);
+quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
+                            const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st);
+
+}  // namespace quoka

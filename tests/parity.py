@@ -1,0 +1,192 @@
+"""Helpers that compare the CUDA path with the CPU oracle stage by stage.
+
+The path is checked as a chain: each stage's CUDA output is validated against the
+oracle within that stage's tie rule, then the CUDA output itself (not the
+oracle's) is fed to the oracle's next stage.  Index work is bit-exact up to ties:
+a rank or a key may differ from the oracle's only where the oracle's own score
+gap is below 1e-4 relative.  Attention outputs on identical indices: bf16 within
+2e-2 max-abs and 2e-3 mean-abs; f32 within 2e-4 / 2e-5.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import quoka_oracle as O
+from paper_2602_08722_b200 import api
+
+REL_TIE = 1e-4
+SCORE_ATOL = 2e-5
+ATTN_TOL = {"bf16": (2e-2, 2e-3), "f32": (2e-4, 2e-5)}
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def check_query_ranks(q_idx_gpu: np.ndarray, cos: np.ndarray, n_retain: int):
+    """q_idx_gpu (n_Q, N), cos (n_Q, C) from the oracle."""
+    n_q, C = cos.shape
+    if C <= n_retain:
+        np.testing.assert_array_equal(q_idx_gpu, np.tile(np.arange(C), (n_q, 1)))
+        return 0
+    swaps = 0
+    for h in range(n_q):
+        g = q_idx_gpu[h].astype(np.int64)
+        assert len(set(g.tolist())) == len(g) and g.min() >= 0 and g.max() < C
+        order = np.argsort(cos[h], kind="stable")
+        want = order[:n_retain]
+        tau = cos[h][order[n_retain - 1]]
+        tol = REL_TIE * abs(tau)
+        chosen = np.zeros(C, bool)
+        chosen[g] = True
+        assert chosen[cos[h] < tau - tol].all(), "a clearly dissimilar query was not retained"
+        assert not chosen[cos[h] > tau + tol].any(), "a clearly similar query was retained"
+        cg = cos[h][g]
+        gaps = np.diff(cg)
+        assert (gaps >= -REL_TIE * np.abs(cg[1:]) - 1e-12).all(), "retained queries out of rank order"
+        swaps += int((g != want).sum())
+    return swaps
+
+
+def check_qbar(qbar_gpu: np.ndarray, qbar_oracle: np.ndarray, dtype: str):
+    diff = np.abs(qbar_gpu - qbar_oracle)
+    if dtype == "bf16":
+        ulp = np.maximum(np.abs(qbar_oracle), 2.0 ** -126) * 2.0 ** -7    # one bf16 ulp is at most 2^-7 relative
+        assert (diff <= ulp).all(), f"Qbar differs by more than one bf16 ulp (max {diff.max()})"
+        assert (diff > 0).mean() < 0.01, "too many Qbar entries rounded differently"
+    else:
+        assert diff.max() <= 1e-6, f"Qbar max abs diff {diff.max()}"
+
+
+def check_key_selection(k_idx_gpu: np.ndarray, scores_oracle: np.ndarray, B: int):
+    """k_idx_gpu (n_KV, >=B); scores_oracle (n_KV, T)."""
+    n_kv, T = scores_oracle.shape
+    diffs = 0
+    for kv in range(n_kv):
+        g = k_idx_gpu[kv, :B].astype(np.int64)
+        assert len(g) == B
+        if B == 0:
+            continue
+        assert (np.diff(g) > 0).all(), "selected rows not ascending / not unique"
+        assert g.min() >= 0 and g.max() < T
+        s = scores_oracle[kv]
+        want = O.select_keys(s[None], B)[0]
+        tau = np.sort(s)[::-1][B - 1]
+        tol = REL_TIE * abs(tau)
+        chosen = np.zeros(T, bool)
+        chosen[g] = True
+        assert chosen[s > tau + tol].all(), "a key clearly above the threshold was dropped"
+        assert not chosen[s < tau - tol].any(), "a key clearly below the threshold was selected"
+        diffs += int(B - np.intersect1d(g, want).size)
+    return diffs
+
+
+def check_attention(out_gpu: np.ndarray, out_oracle: np.ndarray, dtype: str):
+    diff = np.abs(out_gpu - out_oracle)
+    mx, mean = ATTN_TOL[dtype]
+    assert np.isfinite(out_gpu).all()
+    assert diff.max() <= mx, f"attention max abs diff {diff.max()} > {mx}"
+    assert diff.mean() <= mean, f"attention mean abs diff {diff.mean()} > {mean}"
+
+
+class GpuProblem:
+    """Device buffers + params for one ChunkInputs."""
+
+    def __init__(self, inp, n_retain, kv_budget=0, budget_frac=0.0, impl=api.IMPL_AUTO, paged=False,
+                 max_ctx_len=None):
+        dev = "cuda"
+        self.inp = inp
+        self.dtype = inp.dtype
+        self.q = inp.q.to(dev)
+        if paged:
+            self.k = inp.k_pages.to(dev)
+            self.v = inp.v_pages.to(dev)
+            self.block_table = inp.block_table.to(dev)
+        else:
+            self.k = inp.k.to(dev)
+            self.v = inp.v.to(dev)
+            self.block_table = None
+        self.ctx_len = inp.ctx_len.to(dev)
+        self.out = torch.zeros_like(self.q)
+        b, n_q, C, d = self.q.shape
+        n_kv = self.k.shape[1]
+        self.b, self.n_q, self.n_kv, self.C, self.d = b, n_q, n_kv, C, d
+        self.max_ctx = int(inp.ctx_len.max()) if max_ctx_len is None else int(max_ctx_len)
+        self.n_retain, self.kv_budget, self.budget_frac = n_retain, kv_budget, budget_frac
+        self.p = api.make_params(self.q, self.k, self.out, self.ctx_len, n_retain=n_retain, kv_budget=kv_budget,
+                                 budget_frac=budget_frac, max_ctx_len=self.max_ctx, block_table=self.block_table,
+                                 impl=impl)
+        self.N = min(n_retain, C)
+        self.cap = api.quoka_kv_budget_cap(self.p)
+        self.ws = api.alloc_workspace(self.p)
+        self.q_idx = torch.full((b, n_q, self.N), -7, dtype=torch.int32, device=dev)
+        self.qbar = torch.zeros((b, n_kv, self.N, d), dtype=self.q.dtype, device=dev)
+        self.scores = torch.full((b, n_kv, max(self.max_ctx, 1)), float("nan"), dtype=torch.float32, device=dev)
+        self.k_idx = torch.full((b, n_kv, self.cap), -7, dtype=torch.int32, device=dev)
+        self.k_cnt = torch.full((b,), -7, dtype=torch.int32, device=dev)
+        self.lse = torch.zeros((b, n_q, C), dtype=torch.float32, device=dev)
+
+    def run_staged(self):
+        api.quoka_select_queries(self.p, self.q, self.q_idx, self.qbar, self.ws)
+        api.quoka_score_keys(self.p, self.qbar, self.k, self.scores, self.ws)
+        api.quoka_select_keys(self.p, self.scores, self.k_idx, self.k_cnt, self.ws)
+        api.quoka_sparse_attn(self.p, self.q, self.k, self.v, self.k_idx, self.k_cnt, self.out, self.lse, self.ws)
+        torch.cuda.synchronize()
+        assert api.quoka_last_device_status(self.ws) == 0
+
+    def oracle_inputs(self, s):
+        T = int(self.inp.ctx_len[s])
+        q = f64(self.inp.q[s])
+        k = f64(self.inp.k[s, :, : T + self.C])
+        v = f64(self.inp.v[s, :, : T + self.C])
+        return q, k, v, T
+
+
+def check_chain(gp: GpuProblem, attn_rows=None, seed=0):
+    """Validate every stage of a staged run against the oracle.  attn_rows: number of
+    sampled (head, row) pairs per sequence for the attention check (None = all rows)."""
+    stats = dict(rank_swaps=0, key_diffs=0)
+    for s in range(gp.b):
+        q, k, v, T = gp.oracle_inputs(s)
+        B = O.key_budget(T, gp.kv_budget, gp.budget_frac)
+        assert int(gp.k_cnt[s]) == B
+        # stage 1
+        _, cos = O.select_queries(q, gp.n_retain)
+        q_idx = gp.q_idx[s].cpu().numpy()
+        stats["rank_swaps"] += check_query_ranks(q_idx, cos, gp.n_retain)
+        # stage 2 on the GPU's ranks
+        qbar_o = O.aggregate_queries(q, q_idx, gp.n_kv, gp.dtype)
+        qbar_g = f64(gp.qbar[s])
+        check_qbar(qbar_g, qbar_o, gp.dtype)
+        # stage 3 on the GPU's Qbar
+        if T > 0:
+            sc_o = O.score_keys(qbar_g, k, T)
+            sc_g = f64(gp.scores[s, :, :T])
+            assert np.abs(sc_g - sc_o).max() <= SCORE_ATOL, f"score max abs diff {np.abs(sc_g - sc_o).max()}"
+            assert np.abs(sc_g).max() <= 1 + 1e-5
+        else:
+            sc_o = np.zeros((gp.n_kv, 0))
+        # stage 4: band rule against the oracle's scores
+        k_idx = gp.k_idx[s].cpu().numpy()
+        stats["key_diffs"] += check_key_selection(k_idx, sc_o, B)
+        assert (k_idx[:, B:] == -1).all()
+        # exact integer parity of the selection step on the GPU's own fp32 scores
+        if T > 0:
+            want = O.select_keys(f64(gp.scores[s, :, :T]), B)
+            np.testing.assert_array_equal(k_idx[:, :B], want)
+        # stage 5 on the GPU's indices
+        idx_list = [k_idx[kv, :B] for kv in range(gp.n_kv)]
+        out_g = f64(gp.out[s])
+        if attn_rows is None:
+            out_o, lse_o = O.sparse_attention(q, k, v, T, idx_list)
+            check_attention(out_g, out_o, gp.dtype)
+            assert np.abs(f64(gp.lse[s]) - lse_o).max() <= 2e-3
+        else:
+            r = np.random.default_rng(seed + s)
+            heads = r.integers(0, gp.n_q, attn_rows)
+            rows = r.integers(0, gp.C, attn_rows)
+            rows[0], rows[1] = 0, gp.C - 1
+            out_o = O.sparse_attention_rows(q, k, v, T, idx_list, heads, rows)
+            check_attention(out_g[heads, rows], out_o, gp.dtype)
+    return stats

@@ -1,0 +1,225 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import quoka_oracle as O
+from paper_2602_08722_b200 import api, synth
+from tests.parity import GpuProblem, check_attention, check_chain, f64
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [pytest.param(api.IMPL_SIMT, id="simt"), pytest.param(api.IMPL_AUTO, id="auto")]
+
+
+def problem(seed, *, batch=1, n_q=4, n_kv=2, d=128, T=1000, C=300, dtype="bf16", n_retain=24, kv_budget=177,
+            budget_frac=0.0, impl=api.IMPL_AUTO, paged=False, capacity=None, max_ctx_len=None):
+    inp = synth.make_chunk_inputs(seed, batch, n_q, n_kv, d, T, C, dtype, capacity=capacity)
+    if paged:
+        inp = synth.to_paged(inp, seed)
+    return GpuProblem(inp, n_retain, kv_budget, budget_frac, impl=impl, paged=paged, max_ctx_len=max_ctx_len)
+
+
+# ---------------------------------------------------------------- small cases, every stage, all rows
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("name", ["tiny_bf16", "tiny_f32"])
+def test_tiny_config(name, impl):
+    w = synth.WORKLOADS[name]
+    gp = problem(1, n_q=w["n_q"], n_kv=w["n_kv"], d=w["d"], T=w["T"], C=w["C"], dtype=w["dtype"],
+                 n_retain=w["n_retain"], kv_budget=w["kv_budget"], impl=impl)
+    gp.run_staged()
+    check_chain(gp)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("d,dtype", [(128, "bf16"), (64, "bf16"), (128, "f32"), (64, "f32")])
+def test_ragged_sizes(d, dtype, impl):
+    # T, C, N, B all off tile boundaries; several 128-row tiles and a ragged tail everywhere
+    gp = problem(2, n_q=6, n_kv=2, d=d, T=1237, C=333, dtype=dtype, n_retain=37, kv_budget=291, impl=impl)
+    gp.run_staged()
+    check_chain(gp)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("T,C,n_retain,kv_budget", [
+    (0, 200, 16, 64),        # empty cache: pure causal self-attention of the chunk
+    (1, 130, 16, 64),        # one cached key
+    (77, 129, 8, 500),       # budget covers the cache: identity selection, equals dense
+    (500, 40, 64, 100),      # chunk not longer than N_Q: no query sub-selection
+    (300, 1, 4, 50),         # single-query chunk
+    (129, 257, 256, 128),    # N_Q just below C
+])
+def test_degenerate_cases(T, C, n_retain, kv_budget, impl):
+    gp = problem(3, n_q=4, n_kv=2, T=T, C=C, n_retain=n_retain, kv_budget=kv_budget, impl=impl)
+    gp.run_staged()
+    check_chain(gp)
+    if kv_budget >= T:
+        q, k, v, _ = gp.oracle_inputs(0)
+        dense, _ = O.dense_chunk_attention(q, k, v, T)
+        check_attention(f64(gp.out[0]), dense, "bf16")
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("G", [1, 4, 8])
+def test_gqa_ratios(G, impl):
+    gp = problem(4, n_q=8, n_kv=8 // G, T=700, C=260, n_retain=32, kv_budget=0, budget_frac=0.25, impl=impl)
+    gp.run_staged()
+    check_chain(gp)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("paged", [False, True])
+def test_batched_variable_lengths(paged, impl):
+    gp = problem(5, batch=3, n_q=4, n_kv=2, T=[900, 130, 517], C=192, n_retain=16, kv_budget=0, budget_frac=0.12,
+                 impl=impl, paged=paged)
+    gp.run_staged()
+    check_chain(gp)
+
+
+def test_max_ctx_len_may_exceed_every_sequence():
+    gp = problem(6, T=600, C=128, capacity=2048, max_ctx_len=1500, kv_budget=0, budget_frac=0.5)
+    gp.run_staged()
+    check_chain(gp)
+
+
+# ---------------------------------------------------------------- dense kernel, fused call, determinism
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_dense_chunk_attention(dtype, impl):
+    gp = problem(7, n_q=4, n_kv=2, T=777, C=300, dtype=dtype, impl=impl)
+    api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+    torch.cuda.synchronize()
+    q, k, v, T = gp.oracle_inputs(0)
+    want, lse = O.dense_chunk_attention(q, k, v, T)
+    check_attention(f64(gp.out[0]), want, dtype)
+    assert np.abs(f64(gp.lse[0]) - lse).max() <= 2e-3
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("paged", [False, True])
+def test_fused_call_equals_staged_calls(paged, impl):
+    gp = problem(8, batch=2, n_q=8, n_kv=2, T=[1500, 700], C=256, n_retain=32, kv_budget=200, impl=impl, paged=paged)
+    gp.run_staged()
+    staged_out, staged_idx = gp.out.clone(), gp.k_idx.clone()
+    gp.out.zero_()
+    k_idx2 = torch.full_like(gp.k_idx, -9)
+    k_cnt2 = torch.full_like(gp.k_cnt, -9)
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, k_idx2, k_cnt2, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(k_idx2, staged_idx) and torch.equal(k_cnt2, gp.k_cnt)
+    assert torch.equal(gp.out, staged_out)
+    # and without the optional outputs
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged_out)
+    assert api.quoka_last_device_status(gp.ws) == 0
+
+
+def test_fused_call_with_empty_cache():
+    gp = problem(9, T=0, C=150, n_retain=8, kv_budget=32)
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    q, k, v, T = gp.oracle_inputs(0)
+    want, _ = O.dense_chunk_attention(q, k, v, 0)
+    check_attention(f64(gp.out[0]), want, "bf16")
+    assert int(gp.k_cnt[0]) == 0
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_runs_are_bit_identical(impl):
+    gp = problem(10, n_q=8, n_kv=2, T=3000, C=256, n_retain=32, kv_budget=300, impl=impl)
+    gp.run_staged()
+    first = [t.clone() for t in (gp.q_idx, gp.qbar, gp.scores, gp.k_idx, gp.out)]
+    for _ in range(2):
+        gp.run_staged()
+        for a, b in zip(first, (gp.q_idx, gp.qbar, gp.scores, gp.k_idx, gp.out)):
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    gp = problem(11, n_q=8, n_kv=2, T=2000, C=256, n_retain=32, kv_budget=256)
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    want = gp.out.clone()
+    T, C = 2000, 256
+    q_host = gp.inp.q.contiguous().pin_memory()
+    k_new = gp.inp.k[:, :, T:T + C].contiguous().pin_memory()
+    v_new = gp.inp.v[:, :, T:T + C].contiguous().pin_memory()
+    out_host = torch.zeros_like(q_host).pin_memory()
+    gp.k[:, :, T:T + C].zero_()
+    gp.v[:, :, T:T + C].zero_()
+    q_dev = torch.zeros_like(gp.q)
+    gp.out.zero_()
+    ctx_host = gp.inp.ctx_len.clone()
+    api.quoka_prefill_chunk_host(gp.p, ctx_host, q_host, k_new, v_new, out_host, q_dev, gp.k, gp.v, gp.out, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out_host, want.cpu())
+
+
+# ---------------------------------------------------------------- selection step alone: exact integer parity
+@pytest.mark.parametrize("T,B", [(5000, 600), (1024, 1), (1025, 1024), (33, 7), (70000, 8400)])
+def test_select_keys_exact_with_planted_ties(T, B):
+    r = np.random.default_rng(T)
+    s = r.normal(size=(3, T)).astype(np.float32)
+    s[0, :] = np.round(s[0] * 4) / 4            # heavy duplication: many ties at the threshold
+    s[1, ::3] = 0.5
+    s[1, 5] = -0.0
+    s[1, 6] = 0.0
+    inp = synth.make_chunk_inputs(0, 1, 3, 3, 64, T, 8, "bf16")
+    gp = GpuProblem(inp, 4, kv_budget=B)
+    gp.scores[0, :, :T] = torch.from_numpy(s).cuda()
+    api.quoka_select_keys(gp.p, gp.scores, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    want = O.select_keys(s.astype(np.float64), B)
+    np.testing.assert_array_equal(gp.k_idx[0, :, :B].cpu().numpy(), want)
+    assert int(gp.k_cnt[0]) == B
+
+
+# ---------------------------------------------------------------- full-size configurations
+def test_llama8b_32k_full_size():
+    w = synth.WORKLOADS["llama8b_32k"]
+    gp = problem(0, n_q=w["n_q"], n_kv=w["n_kv"], d=w["d"], T=w["T"], C=w["C"], n_retain=w["n_retain"],
+                 kv_budget=w["kv_budget"])
+    gp.run_staged()
+    stats = check_chain(gp, attn_rows=256)
+    staged = gp.out.clone()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(staged, gp.out)
+    print("llama8b_32k parity stats", stats)
+
+
+def test_long_128k_full_size():
+    w = synth.WORKLOADS["long_128k"]
+    gp = problem(0, n_q=w["n_q"], n_kv=w["n_kv"], d=w["d"], T=w["T"], C=w["C"], n_retain=w["n_retain"],
+                 kv_budget=w["kv_budget"])
+    gp.run_staged()
+    stats = check_chain(gp, attn_rows=128)
+    print("long_128k parity stats", stats)
+
+
+def test_serving_mix_paged_full_size():
+    w = synth.WORKLOADS["serving_mix"]
+    lens = synth.serving_mix_ctx_lens(0, w["batch"])
+    gp = problem(0, batch=w["batch"], n_q=w["n_q"], n_kv=w["n_kv"], d=w["d"], T=lens, C=w["C"],
+                 n_retain=w["n_retain"], kv_budget=0, budget_frac=w["budget_frac"], paged=True)
+    gp.run_staged()
+    stats = check_chain(gp, attn_rows=64)
+    print("serving_mix parity stats", stats)
+
+
+SWEEP_BASE = dict(budget_frac=0.12, C=2048, d=128, G=4, n_retain=128)
+SWEEP_POINTS = [dict()] + [dict(budget_frac=f) for f in (0.05, 0.25, 0.5)] + [dict(C=c) for c in (512, 8192)] + \
+    [dict(d=64)] + [dict(G=g) for g in (1, 8)] + [dict(n_retain=n) for n in (32, 512)] + \
+    [dict(budget_frac=0.05, C=512, d=64, G=8, n_retain=32), dict(budget_frac=0.5, C=8192, d=128, G=1, n_retain=512),
+     dict(budget_frac=0.5, C=512, d=64, G=1, n_retain=512), dict(budget_frac=0.05, C=8192, d=128, G=8, n_retain=32)]
+
+
+@pytest.mark.parametrize("pt", SWEEP_POINTS, ids=lambda p: "-".join(f"{k}{v}" for k, v in p.items()) or "base")
+def test_sweep_points_32k(pt):
+    c = dict(SWEEP_BASE, **pt)
+    gp = problem(0, n_q=32, n_kv=32 // c["G"], d=c["d"], T=32768, C=c["C"], n_retain=c["n_retain"], kv_budget=0,
+                 budget_frac=c["budget_frac"])
+    gp.run_staged()
+    check_chain(gp, attn_rows=64)
