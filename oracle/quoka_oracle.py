@@ -134,7 +134,7 @@ def score_keys(qbar, k, T):
     kc = np.asarray(k, dtype=np.float64)[:, :T, :]
     kn = np.maximum(np.sqrt((kc * kc).sum(axis=2, keepdims=True)), EPS)
     k_hat = kc / kn
-    S = np.einsum("hnd,htd->hnt", qbar, k_hat)                # (n_KV, N, T)
+    S = qbar @ np.swapaxes(k_hat, 1, 2)                       # (n_KV, N, T)
     if S.shape[1] == 0:
         return np.full((kc.shape[0], T), -np.inf)
     return S.max(axis=1)

@@ -52,8 +52,10 @@ def check_query_ranks(q_idx_gpu: np.ndarray, cos: np.ndarray, n_retain: int):
 def check_qbar(qbar_gpu: np.ndarray, qbar_oracle: np.ndarray, dtype: str):
     diff = np.abs(qbar_gpu - qbar_oracle)
     if dtype == "bf16":
-        ulp = np.maximum(np.abs(qbar_oracle), 2.0 ** -126) * 2.0 ** -7    # one bf16 ulp is at most 2^-7 relative
-        assert (diff <= ulp).all(), f"Qbar differs by more than one bf16 ulp (max {diff.max()})"
+        # one bf16 ulp is at most 2^-7 relative; entries that nearly cancel carry the fp32 accumulation
+        # error of their O(0.1) terms (a few 1e-8) on top, which near zero exceeds their own ulp
+        ulp = np.abs(qbar_oracle) * 2.0 ** -7 + 2e-7
+        assert (diff <= ulp).all(), f"Qbar differs by more than one bf16 ulp (max excess {(diff - ulp).max()})"
         assert (diff > 0).mean() < 0.01, "too many Qbar entries rounded differently"
     else:
         assert diff.max() <= 1e-6, f"Qbar max abs diff {diff.max()}"
@@ -161,7 +163,8 @@ def check_chain(gp: GpuProblem, attn_rows=None, seed=0):
         check_qbar(qbar_g, qbar_o, gp.dtype)
         # stage 3 on the GPU's Qbar
         if T > 0:
-            sc_o = O.score_keys(qbar_g, k, T)
+            # one KV head at a time: the oracle materialises the (N, T) score matrix
+            sc_o = np.concatenate([O.score_keys(qbar_g[kv:kv + 1], k[kv:kv + 1], T) for kv in range(gp.n_kv)])
             sc_g = f64(gp.scores[s, :, :T])
             assert np.abs(sc_g - sc_o).max() <= SCORE_ATOL, f"score max abs diff {np.abs(sc_g - sc_o).max()}"
             assert np.abs(sc_g).max() <= 1 + 1e-5
