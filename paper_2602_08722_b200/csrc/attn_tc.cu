@@ -1,10 +1,418 @@
-// Placeholder until the tcgen05 attention kernel lands: reports "not covered" so the scalar kernel runs.
+// Flash-style attention on the 5th-generation tensor cores over
+//   [selected cached rows | the chunk's own causal rows]      (Algorithm 2's attention line, Eq. 2)
+// or, without an index list, over every cached row (Eq. 2, dense chunk attention).  bf16 in, fp32
+// softmax and accumulation, P rounded to bf16 for the PV product.
+//
+// One CTA owns 256 consecutive chunk rows of one query head as two 128-row Q tiles (A, B) and walks
+// the key tiles (128 keys) once for both.  Roles:
+//   warps 0-3 / 4-7  softmax of Q tile A / B: one thread per query row, S read from tensor memory,
+//                    running max / sum in registers, P written back to tensor memory over S,
+//                    lazy rescale of the O accumulator (only when the max grew by more than 2^8),
+//                    final normalisation and the global store.
+//   warps 8-11       loaders: every K / V row of a tile is fetched with 16-byte cp.async straight
+//                    into the 128-byte-swizzled layout the MMA descriptors expect.  The row address
+//                    comes from the selected-index list (the gather), the chunk offset, or the page
+//                    table, so no compacted copy of K or V is ever made; rows past the end are
+//                    zero-filled.
+//   warp 12          MMA issuer (one thread): S = Q K^T (both operands in shared memory) and
+//                    O += P V (P from tensor memory, V in shared memory, MN-major).
+// Tensor memory (512 columns): S_A | S_B | O_A | O_B, P aliasing the first 64 columns of its S.
+// K and V tiles share one ring of shared-memory slots in the order K0 V0 K1 V1 ...
+#include "sm100_ptx.cuh"
 #include "tensor_kernels.cuh"
 
 namespace quoka {
-bool attn_tc_supported(const quoka_params*) { return false; }
-quoka_status launch_attn_tc(const quoka_params*, const DevParams&, const void*, const void*, const void*,
-                            const int32_t*, const int32_t*, void*, float*, cudaStream_t) {
-  return QUOKA_ERR_UNSUPPORTED;
+
+using namespace ptx;
+
+constexpr int kAttnThreads = 13 * 32;
+constexpr int kQTile = 128;
+constexpr int kKeyTile = 128;
+constexpr int kSlots = 5;
+constexpr int kLoaderLag = 2;               // key/value tiles in flight per loader thread
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
+
+bool encode_kv_tensor_map(CUtensorMap* out, const quoka_params* p, const void* cache, uint32_t box_rows);
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
+
+struct AttnGeom {
+  int T, cnt, n_sel;        // cached length, selected rows, selected tiles (sparse); cnt = T, n_sel unused (dense)
+  int n_a, n_b, n_max;      // key tiles Q tile A / B take part in, and their maximum
+};
+
+template <bool SPARSE>
+__device__ __forceinline__ AttnGeom make_geom(const DevParams& P, int s, int r0, const int32_t* k_cnt) {
+  AttnGeom g;
+  g.T = __ldg(P.ctx_len + s);
+  const int C = P.chunk;
+  const bool b_active = r0 + kQTile < C;
+  if (SPARSE) {
+    g.cnt = __ldg(k_cnt + s);
+    g.n_sel = (g.cnt + kKeyTile - 1) / kKeyTile;
+    g.n_a = g.n_sel + r0 / kQTile + 1;
+    g.n_b = b_active ? g.n_a + 1 : 0;
+  } else {
+    g.cnt = g.T;
+    g.n_sel = 0;
+    const int last_a = min(r0 + kQTile - 1, C - 1), last_b = min(r0 + 2 * kQTile - 1, C - 1);
+    g.n_a = (g.T + last_a) / kKeyTile + 1;
+    g.n_b = b_active ? (g.T + last_b) / kKeyTile + 1 : 0;
+  }
+  g.n_max = max(g.n_a, g.n_b);
+  return g;
+}
+
+// Number of visible columns of key tile j for chunk row `row` (columns [0, lim) are visible).
+template <bool SPARSE>
+__device__ __forceinline__ int visible_cols(const AttnGeom& g, int j, int row) {
+  int lim;
+  if (SPARSE) {
+    if (j < g.n_sel) lim = g.cnt - j * kKeyTile;
+    else lim = row - (j - g.n_sel) * kKeyTile + 1;
+  } else {
+    lim = g.T + row - j * kKeyTile + 1;
+  }
+  return max(0, min(kKeyTile, lim));
+}
+
+template <int HALVES, bool SPARSE>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv_bfloat16* __restrict__ kc,
+               const __nv_bfloat16* __restrict__ vc, const int32_t* __restrict__ k_idx,
+               const int32_t* __restrict__ k_cnt, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+  constexpr int D = HALVES * 64;
+  constexpr uint32_t kHalfBytes = 128 * 128;                 // 128 rows x 128 B
+  constexpr uint32_t kTileBytes = HALVES * kHalfBytes;       // one Q / K / V tile
+  constexpr uint32_t S_COL[2] = {0, 128}, O_COL[2] = {256, 384};
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* q_smem = smem;                               // [2][HALVES][128][128 B]
+  unsigned char* kv_smem = smem + 2 * kTileBytes;             // [kSlots][HALVES][128][128 B]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(kv_smem + (size_t)kSlots * kTileBytes);
+  uint64_t* kv_full = bars;                 // [kSlots]  4 loader warps arrive
+  uint64_t* kv_empty = bars + kSlots;       // [kSlots]  MMA commit
+  uint64_t* s_full = bars + 2 * kSlots;     // [2]       MMA commit
+  uint64_t* p_full = s_full + 2;            // [2]       4 softmax warps arrive
+  uint64_t* o_full = p_full + 2;            // [2]       MMA commit after the last PV
+  uint64_t* q_full = o_full + 2;            // TMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_full + 1);
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WaitCtx wc{&abort_flag, P.status};
+  const int s = blockIdx.z, h = blockIdx.y, kv = h / P.group;
+  const int rb = gridDim.x - 1 - blockIdx.x;                  // heaviest row blocks first
+  const int r0 = rb * 2 * kQTile;
+  const AttnGeom g = make_geom<SPARSE>(P, s, r0, k_cnt);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < kSlots; ++i) { mbar_init(&kv_full[i], 4); mbar_init(&kv_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); mbar_init(&o_full[i], 1); }
+    mbar_init(q_full, 1);
+    fence_mbar_init();
+    tma_prefetch_desc(&tm_q);
+  }
+  if (warp == 12) tmem_alloc(tmem_slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp < 8) {
+    // ================================================================== softmax + epilogue
+    const int x = warp >> 2;                                  // Q tile A (0) or B (1)
+    const int n_tiles = x ? g.n_b : g.n_a;
+    const int quarter = warp & 3;
+    const int row_in_tile = quarter * 32 + lane;
+    const int row = r0 + x * kQTile + row_in_tile;            // chunk row
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t s_addr = lane_addr + S_COL[x], o_addr = lane_addr + O_COL[x];
+    const float scale_log2 = P.scale * 1.4426950408889634f;
+    float m_run = -INFINITY, l_run = 0.f;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      if (!mbar_wait(&s_full[x], phase, wc)) { ok = false; break; }
+      phase ^= 1;
+      tc_fence_after();
+      const int lim = visible_cols<SPARSE>(g, j, row);
+      const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
+      // ---- pass 1: row maximum of the raw logits
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(s_addr + c * 32, r);
+        tmem_wait_ld();
+        if (masked) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) if (c * 32 + i < lim) mx = fmaxf(mx, __uint_as_float(r[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+        }
+      }
+      const float m_tile = mx * scale_log2;
+      // ---- lazy rescale of the accumulator: only when some row's maximum grew by more than the threshold
+      const bool grow = m_tile > m_run + kRescaleThreshold;
+      if (__any_sync(0xFFFFFFFFu, grow)) {
+        const float m_new = fmaxf(m_run, m_tile);
+        if (j > 0) {
+          const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
+          l_run *= alpha;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(o_addr + c * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st32(o_addr + c * 32, r);
+          }
+          tmem_wait_st();
+        }
+        m_run = m_new;
+      }
+      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+      // ---- pass 2: p = 2^(s*scale - m), row sum, bf16 P over the first 64 columns of S
+      float psum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(s_addr + c * 32, r);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), scale_log2, -m_use));
+          float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, -m_use));
+          if (masked) {
+            if (c * 32 + 2 * i >= lim) p0 = 0.f;
+            if (c * 32 + 2 * i + 1 >= lim) p1 = 0.f;
+          }
+          psum += p0 + p1;
+          const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+          pk[i] = *reinterpret_cast<const uint32_t*>(&b2);
+        }
+        tmem_st16(s_addr + c * 16, pk);
+      }
+      l_run += psum;
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&p_full[x]);
+    }
+    // ---- epilogue: O / l -> bf16 -> global
+    if (ok && n_tiles > 0 && mbar_wait(&o_full[x], 0, wc)) {
+      tc_fence_after();
+      const float inv = 1.f / l_run;
+      const bool store = row < P.chunk;
+      __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(o_addr + c * 32, r);
+        tmem_wait_ld();
+        if (store) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
+                                                               __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
+              w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      if (store && lse)
+        lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    }
+  } else if (warp < 12) {
+    // ================================================================== K / V row loaders (gather)
+    const int lt = threadIdx.x - 8 * 32;                      // 0..127
+    constexpr int PIECES = D / 8;                             // 16-byte pieces per row (16 or 8)
+    constexpr int ROWS_PER_PASS = 128 / PIECES;               // rows the 128 loader threads cover at once
+    const int c16 = lt % PIECES;                              // this thread's piece of the row
+    const int rsub = lt / PIECES;
+    const int32_t* idx = SPARSE ? k_idx + ((long long)s * P.n_kv + kv) * P.budget_cap : nullptr;
+    const int n_items = 2 * g.n_max;
+    uint32_t phase = 0;
+    int slot = 0, done_slot = 0;
+    bool ok = true;
+    const uint32_t kv_base = smem_u32(kv_smem);
+    for (int it = 0; it < n_items; ++it) {
+      if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) { ok = false; break; }
+      const int j = it >> 1;
+      const __nv_bfloat16* src_base = (it & 1) ? vc : kc;
+      const uint32_t dst_tile = kv_base + slot * kTileBytes;
+      {
+#pragma unroll 4
+        for (int rr = rsub; rr < kKeyTile; rr += ROWS_PER_PASS) {
+          int t;
+          bool valid;
+          if (SPARSE) {
+            if (j < g.n_sel) {
+              const int u = j * kKeyTile + rr;
+              valid = u < g.cnt;
+              t = valid ? __ldg(idx + u) : 0;
+            } else {
+              const int pos = (j - g.n_sel) * kKeyTile + rr;
+              valid = pos < P.chunk;
+              t = g.T + pos;
+            }
+          } else {
+            t = j * kKeyTile + rr;
+            valid = t < g.T + P.chunk;
+          }
+          const __nv_bfloat16* src = valid ? src_base + kv_row_offset(P, s, kv, t) + c16 * 8 : src_base;
+          const uint32_t dst = dst_tile + (c16 >> 3) * kHalfBytes + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
+          cp_async_16(dst, src, valid);
+        }
+      }
+      cp_async_commit();
+      if (it >= kLoaderLag) {
+        cp_async_wait<kLoaderLag>();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&kv_full[done_slot]);
+        if (++done_slot == kSlots) done_slot = 0;
+      }
+      if (++slot == kSlots) { slot = 0; phase ^= 1; }
+    }
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (ok) {
+      const int pending = n_items < kLoaderLag ? n_items : kLoaderLag;
+      for (int i = 0; i < pending; ++i) {
+        if (lane == 0) mbar_arrive(&kv_full[done_slot]);
+        if (++done_slot == kSlots) done_slot = 0;
+      }
+    }
+  } else if (lane == 0) {
+    // ================================================================== MMA issuer (warp 12, one thread)
+    mbar_arrive_expect_tx(q_full, 2 * kTileBytes);
+    for (int x = 0; x < 2; ++x)
+      for (int hh = 0; hh < HALVES; ++hh)
+        tma_load_4d(q_smem + x * kTileBytes + hh * kHalfBytes, &tm_q, q_full, hh * 64, r0 + x * kQTile, h, s);
+    const uint32_t idesc_qk = idesc_bf16_f32(128, kKeyTile, false, false);
+    const uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
+    const uint32_t q_base = smem_u32(q_smem), kv_base = smem_u32(kv_smem);
+    int slot = 0;
+    uint32_t kv_phase = 0;
+    uint32_t p_phase[2] = {0, 0};
+    int k_slot = -1, v_slot = -1;
+    bool ok = mbar_wait(q_full, 0, wc);
+    auto acquire = [&]() -> int {           // next ring item (K or V) becomes readable
+      if (!mbar_wait(&kv_full[slot], kv_phase, wc)) { ok = false; return 0; }
+      tc_fence_after();
+      const int got = slot;
+      if (++slot == kSlots) { slot = 0; kv_phase ^= 1; }
+      return got;
+    };
+    auto issue_qk = [&](int x, int ks) {
+#pragma unroll
+      for (int hh = 0; hh < HALVES; ++hh)
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          const uint64_t a = smem_desc_sw128(q_base + x * kTileBytes + hh * kHalfBytes + kk * 32, 16, 1024);
+          const uint64_t b = smem_desc_sw128(kv_base + ks * kTileBytes + hh * kHalfBytes + kk * 32, 16, 1024);
+          mma_ss(tmem_base + S_COL[x], a, b, idesc_qk, (hh | kk) ? 1u : 0u);
+        }
+      mma_commit(&s_full[x]);
+    };
+    auto issue_pv = [&](int x, int vs, int j) {
+      if (!mbar_wait(&p_full[x], p_phase[x], wc)) { ok = false; return; }
+      p_phase[x] ^= 1;
+      tc_fence_after();
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {       // 16 keys per MMA: 8 packed columns of P, 16 rows of V
+        const uint64_t b = smem_desc_sw128(kv_base + vs * kTileBytes + kk * 2048, kHalfBytes, 1024);
+        mma_ts(tmem_base + O_COL[x], tmem_base + S_COL[x] + kk * 8, b, idesc_pv, (j | kk) ? 1u : 0u);
+      }
+    };
+    if (ok && g.n_max > 0) {
+      k_slot = acquire();
+      if (ok) {
+        if (g.n_a > 0) issue_qk(0, k_slot);
+        if (g.n_b > 0) issue_qk(1, k_slot);
+        mma_commit(&kv_empty[k_slot]);
+      }
+      for (int j = 0; ok && j < g.n_max; ++j) {
+        v_slot = acquire();
+        if (!ok) break;
+        const bool more = j + 1 < g.n_max;
+        if (j < g.n_a) {
+          issue_pv(0, v_slot, j);
+          if (!ok) break;
+          if (j + 1 == g.n_a) mma_commit(&o_full[0]);
+        }
+        if (more) {
+          k_slot = acquire();
+          if (!ok) break;
+          if (j + 1 < g.n_a) issue_qk(0, k_slot);
+        }
+        if (j < g.n_b) {
+          issue_pv(1, v_slot, j);
+          if (!ok) break;
+          if (j + 1 == g.n_b) mma_commit(&o_full[1]);
+        }
+        mma_commit(&kv_empty[v_slot]);
+        if (more) {
+          if (j + 1 < g.n_b) issue_qk(1, k_slot);
+          mma_commit(&kv_empty[k_slot]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 12) tmem_dealloc(tmem_base, 512);
+}
+
+// ---------------------------------------------------------------------------------------------- host
+bool attn_tc_supported(const quoka_params* p) {
+  if (p->dtype != QUOKA_BF16) return false;
+  return true;
+}
+
+quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
+                            const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st) {
+  CUtensorMap tm_q;
+  {
+    const uint64_t dims[4] = {(uint64_t)P.d, (uint64_t)P.chunk, (uint64_t)P.n_q, (uint64_t)P.batch};
+    const uint64_t strides[3] = {(uint64_t)P.q_st * 2, (uint64_t)P.q_sh * 2, (uint64_t)P.q_sb * 2};
+    const uint32_t box[4] = {64, 128, 1, 1};
+    if (!encode_tensor_map_bf16(&tm_q, q, 4, dims, strides, box)) return QUOKA_ERR_CUDA;
+  }
+  const int halves = P.d / 64;
+  const size_t tile = (size_t)halves * 128 * 128;
+  const size_t smem = 1024 + (2 + kSlots) * tile + 512;
+  dim3 grid((P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.n_q, P.batch);
+  const bool sparse = k_idx != nullptr;
+  cudaError_t e = cudaSuccess;
+#define QUOKA_ATTN_TC(H, S)                                                                                      \
+  do {                                                                                                           \
+    e = cudaFuncSetAttribute(attn_tc_kernel<H, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
+    if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                 \
+    attn_tc_kernel<H, S><<<grid, kAttnThreads, smem, st>>>(P, tm_q, (const __nv_bfloat16*)k,                     \
+                                                           (const __nv_bfloat16*)v, k_idx, k_cnt,                \
+                                                           (__nv_bfloat16*)out, lse);                            \
+  } while (0)
+  if (halves == 2) { if (sparse) QUOKA_ATTN_TC(2, true); else QUOKA_ATTN_TC(2, false); }
+  else { if (sparse) QUOKA_ATTN_TC(1, true); else QUOKA_ATTN_TC(1, false); }
+#undef QUOKA_ATTN_TC
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? QUOKA_OK : QUOKA_ERR_CUDA;
+}
+
 }  // namespace quoka
