@@ -58,7 +58,8 @@ typedef enum {
   QUOKA_ERR_UNSUPPORTED = 2,  /* head_dim not in {64,128}, page_size not in {0,64}, chunk_len > 8192 with selection */
   QUOKA_ERR_WORKSPACE = 3,    /* workspace pointer null / misaligned / smaller than quoka_workspace_size */
   QUOKA_ERR_CUDA = 4,         /* a CUDA runtime or driver call failed (launch, tensor-map encode) */
-  QUOKA_ERR_TIMEOUT = 5       /* device status word: a bounded wait inside a kernel ran out */
+  QUOKA_ERR_TIMEOUT = 5,      /* device status word: a bounded wait inside a kernel ran out */
+  QUOKA_ERR_STATIC_LIMIT = 6  /* quoka_prefill_chunk_static: the problem needs more scratch than the built-in array */
 } quoka_status;
 
 typedef enum { QUOKA_BF16 = 0, QUOKA_F32 = 1 } quoka_dtype;
@@ -162,6 +163,29 @@ quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_
                                       const void* q_host, const void* k_new_host, const void* v_new_host,
                                       void* out_host, void* q_dev, void* k_cache, void* v_cache, void* out_dev,
                                       void* ws, size_t ws_bytes, void* stream);
+
+/* (The paper has no counterpart of this call: it is a deployment variant of quoka_prefill_chunk.)
+ * The same loop body for callers that cannot allocate device memory and so have no workspace to
+ * pass: a process whose KV-cache pool already owns all of HBM, or a latency-critical loop in which
+ * cudaMalloc/cudaFree (which synchronise the device) are forbidden.  The intermediates live in an
+ * array of QUOKA_STATIC_SCRATCH_BYTES that is part of the library image; every GPU that loads the
+ * library holds that much memory until the process exits.  Inputs and outputs are still the
+ * caller's.  The call allocates nothing and frees nothing.
+ *   - Problems whose quoka_workspace_size exceeds QUOKA_STATIC_SCRATCH_BYTES are refused with
+ *     QUOKA_ERR_STATIC_LIMIT before anything is launched (for scale: 32 q / 8 kv heads, d 128,
+ *     131072 cached rows, N_Q 256 needs about 5.1 MiB; a batch of 8 at 65536 rows does not fit).
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current); make that first call before any stream capture begins.
+ *   - All calls in the process share the one array per device, and it keeps the previous call's
+ *     contents.  The status word is cleared at the start of every call; nothing else needs to start
+ *     at zero.  Two calls whose work overlaps on the same GPU (different streams, or different host
+ *     threads) race on the array: serialise them.
+ *   - A timed-out device wait cannot be read back through quoka_last_device_status, which needs
+ *     the workspace pointer; the outputs of such a call are undefined. */
+#define QUOKA_STATIC_SCRATCH_BYTES (8u << 20)
+quoka_status quoka_prefill_chunk_static(const quoka_params* p, const void* q, const void* k_cache,
+                                        const void* v_cache, void* out, int32_t* k_idx_out, int32_t* k_cnt_out,
+                                        void* stream);
 
 /* Copies the device status word of `ws` to the host (synchronises `stream`) and
  * clears it.  *status_out is a quoka_status. */

@@ -15,14 +15,15 @@ import torch
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libquoka.so")
 _lib = None
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_STATIC_LIMIT = range(7)
+STATIC_SCRATCH_BYTES = 8 << 20
 BF16, F32 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "quoka_kv_budget_cap", "quoka_workspace_size", "quoka_select_queries", "quoka_score_keys",
     "quoka_select_keys", "quoka_sparse_attn", "quoka_dense_chunk_attn", "quoka_prefill_chunk",
-    "quoka_prefill_chunk_host", "quoka_last_device_status", "quoka_status_string", "quoka_launch_count",
+    "quoka_prefill_chunk_host", "quoka_prefill_chunk_static", "quoka_last_device_status", "quoka_status_string", "quoka_launch_count",
 ]
 
 
@@ -70,6 +71,7 @@ def load():
     lib.quoka_dense_chunk_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.quoka_prefill_chunk.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.quoka_prefill_chunk_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.quoka_prefill_chunk_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
     lib.quoka_last_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
     for name in EXPORTS:
         if name not in ("quoka_status_string", "quoka_launch_count"):
@@ -182,6 +184,14 @@ def quoka_prefill_chunk_host(p, ctx_len_host, q_host, k_new_host, v_new_host, ou
                                            _ptr(v_new_host), _ptr(out_host), _ptr(q_dev), _ptr(k_cache),
                                            _ptr(v_cache), _ptr(out_dev), _ptr(ws), ws.numel(), _stream(stream)),
            "quoka_prefill_chunk_host")
+
+
+def quoka_prefill_chunk_static(p, q, k_cache, v_cache, out, k_idx_out, k_cnt_out, stream=None):
+    """The fused call on the library's built-in scratch array: for callers that cannot allocate a
+    workspace.  Raises QuokaError(ERR_STATIC_LIMIT) when the problem does not fit the array."""
+    _check(load().quoka_prefill_chunk_static(C.byref(p), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out),
+                                             _ptr(k_idx_out), _ptr(k_cnt_out), _stream(stream)),
+           "quoka_prefill_chunk_static")
 
 
 def quoka_last_device_status(ws, stream=None) -> int:

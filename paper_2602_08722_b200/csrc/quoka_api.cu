@@ -290,6 +290,7 @@ const char* quoka_status_string(quoka_status s) {
     case QUOKA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case QUOKA_ERR_CUDA: return "CUDA call failed";
     case QUOKA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case QUOKA_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in static array holds";
     default: return "unknown status";
   }
 }
