@@ -198,6 +198,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused-only", action="store_true",
+                    help="only the timed fused steps (for profiler captures): no per-kernel, e2e or CPU legs")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -307,6 +309,13 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_us = float(t.item())
     us_per_chunk = total_us / (args.steps * world)       # chunks processed by all ranks / time
+
+    if args.fused_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": round(us_per_chunk, 2), "unit": UNIT, "n_gpus": world,
+                              "steps": args.steps, "warmup": args.warmup, "config": config, "gpu_launches": launches,
+                              "note": "fused-only run (profiling aid); not a bench line"}))
+        return 0
 
     # ---- per-kernel timings through the staged entry points (each alone, L2 flushed between launches)
     ksteps = max(5, min(args.steps, 20))

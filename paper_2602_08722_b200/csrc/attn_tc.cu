@@ -29,7 +29,7 @@ constexpr int kAttnThreads = 13 * 32;
 constexpr int kQTile = 128;
 constexpr int kKeyTile = 128;
 constexpr int kSlots = 5;
-constexpr int kLoaderLag = 2;               // key/value tiles in flight per loader thread
+constexpr int kLoaderLag = 3;               // key/value tiles in flight per loader thread
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
 bool encode_kv_tensor_map(CUtensorMap* out, const quoka_params* p, const void* cache, uint32_t box_rows);
@@ -144,7 +144,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       const int lim = visible_cols<SPARSE>(g, j, row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
       // ---- pass 1: row maximum of the raw logits
-      float mx = -INFINITY;
+      float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
@@ -152,12 +152,13 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         tmem_wait_ld();
         if (masked) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) if (c * 32 + i < lim) mx = fmaxf(mx, __uint_as_float(r[i]));
+          for (int i = 0; i < 32; ++i) if (c * 32 + i < lim) mxa[i & 3] = fmaxf(mxa[i & 3], __uint_as_float(r[i]));
         } else {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+          for (int i = 0; i < 32; ++i) mxa[i & 3] = fmaxf(mxa[i & 3], __uint_as_float(r[i]));
         }
       }
+      const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
       const float m_tile = mx * scale_log2;
       // ---- lazy rescale of the accumulator: only when some row's maximum grew by more than the threshold
       const bool grow = m_tile > m_run + kRescaleThreshold;
@@ -181,7 +182,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       }
       const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
       // ---- pass 2: p = 2^(s*scale - m), row sum, bf16 P over the first 64 columns of S
-      float psum = 0.f;
+      float psa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
@@ -196,13 +197,13 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
             if (c * 32 + 2 * i >= lim) p0 = 0.f;
             if (c * 32 + 2 * i + 1 >= lim) p1 = 0.f;
           }
-          psum += p0 + p1;
+          psa[i & 3] += p0 + p1;
           const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
           pk[i] = *reinterpret_cast<const uint32_t*>(&b2);
         }
         tmem_st16(s_addr + c * 16, pk);
       }
-      l_run += psum;
+      l_run += (psa[0] + psa[1]) + (psa[2] + psa[3]);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
@@ -244,41 +245,56 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     const int c16 = lt % PIECES;                              // this thread's piece of the row
     const int rsub = lt / PIECES;
     const int32_t* idx = SPARSE ? k_idx + ((long long)s * P.n_kv + kv) * P.budget_cap : nullptr;
+    constexpr int RPT = kKeyTile / ROWS_PER_PASS;             // rows per thread per tile (16 or 8)
     const int n_items = 2 * g.n_max;
     uint32_t phase = 0;
     int slot = 0, done_slot = 0;
     bool ok = true;
     const uint32_t kv_base = smem_u32(kv_smem);
+    // Element offset of each of this thread's rows of key tile j (-1 = past the end: zero fill).  The index
+    // list and the page table are read here, one tile ahead of the copies that use them.
+    auto row_offsets = [&](int j, long long (&off)[RPT]) {
+      int t[RPT];
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) {
+        const int rr = rsub + i * ROWS_PER_PASS;
+        if (SPARSE) {
+          if (j < g.n_sel) {
+            const int u = j * kKeyTile + rr;
+            t[i] = u < g.cnt ? __ldg(idx + u) : -1;
+          } else {
+            const int pos = (j - g.n_sel) * kKeyTile + rr;
+            t[i] = pos < P.chunk ? g.T + pos : -1;
+          }
+        } else {
+          const int tt = j * kKeyTile + rr;
+          t[i] = tt < g.T + P.chunk ? tt : -1;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) off[i] = t[i] >= 0 ? kv_row_offset(P, s, kv, t[i]) + c16 * 8 : -1;
+    };
+    long long off_cur[RPT], off_next[RPT];
+    if (g.n_max > 0) row_offsets(0, off_cur);
     for (int it = 0; it < n_items; ++it) {
       if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) { ok = false; break; }
       const int j = it >> 1;
       const __nv_bfloat16* src_base = (it & 1) ? vc : kc;
-      const uint32_t dst_tile = kv_base + slot * kTileBytes;
-      {
-#pragma unroll 4
-        for (int rr = rsub; rr < kKeyTile; rr += ROWS_PER_PASS) {
-          int t;
-          bool valid;
-          if (SPARSE) {
-            if (j < g.n_sel) {
-              const int u = j * kKeyTile + rr;
-              valid = u < g.cnt;
-              t = valid ? __ldg(idx + u) : 0;
-            } else {
-              const int pos = (j - g.n_sel) * kKeyTile + rr;
-              valid = pos < P.chunk;
-              t = g.T + pos;
-            }
-          } else {
-            t = j * kKeyTile + rr;
-            valid = t < g.T + P.chunk;
-          }
-          const __nv_bfloat16* src = valid ? src_base + kv_row_offset(P, s, kv, t) + c16 * 8 : src_base;
-          const uint32_t dst = dst_tile + (c16 >> 3) * kHalfBytes + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
-          cp_async_16(dst, src, valid);
-        }
+      const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) {
+        const int rr = rsub + i * ROWS_PER_PASS;
+        const bool valid = off_cur[i] >= 0;
+        const uint32_t dst = dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
+        cp_async_16(dst, valid ? src_base + off_cur[i] : src_base, valid);
       }
       cp_async_commit();
+      if (!(it & 1)) {
+        if (j + 1 < g.n_max) row_offsets(j + 1, off_next);    // in flight while the V copies are issued
+      } else {
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) off_cur[i] = off_next[i];
+      }
       if (it >= kLoaderLag) {
         cp_async_wait<kLoaderLag>();
         fence_proxy_async_smem();

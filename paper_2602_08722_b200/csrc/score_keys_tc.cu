@@ -95,7 +95,6 @@ template <int HALVES>   // head_dim / 64
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k, float* __restrict__ scores) {
-  constexpr int D = HALVES * 64;
   constexpr uint32_t kHalfBytes = kTileKeys * 128;             // one 64-column half of a K tile
   constexpr uint32_t kStageBytes = HALVES * kHalfBytes;
   extern __shared__ unsigned char smem_raw[];
@@ -219,7 +218,7 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
     for (; w.valid(); w.next(P)) {
       if (!mbar_wait(&full[stage], phase, wc)) break;
       // |k|^2 from the tile in shared memory (rotated 16-byte reads: conflict-free)
-      float nn = 0.f;
+      float nacc[4] = {0.f, 0.f, 0.f, 0.f};                 // independent partial sums: no 256-deep FMA chain
       const unsigned char* krow = k_smem + (size_t)stage * kStageBytes + row * 128;
 #pragma unroll
       for (int h = 0; h < HALVES; ++h) {
@@ -230,20 +229,41 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float a = __uint_as_float(wds[i] << 16), b = __uint_as_float(wds[i] & 0xFFFF0000u);
-            nn = fmaf(a, a, nn);
-            nn = fmaf(b, b, nn);
+            nacc[i] = fmaf(a, a, nacc[i]);
+            nacc[i] = fmaf(b, b, nacc[i]);
           }
         }
       }
+      const float nn = (nacc[0] + nacc[1]) + (nacc[2] + nacc[3]);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);
       if (!mbar_wait(&acc_full[slot], acc_phase, wc)) break;
       tc_fence_after();
-      float best = -INFINITY;
+      float bacc[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       for (int p = 0; p < A.n_parts; ++p) {
         const int n_mma = (p == A.n_parts - 1) ? (A.n_pad - p * 256) : 256;
         const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((A.n_parts == 1 ? slot : p) * 256);
         int c0 = 0;
+        for (; c0 + 64 <= n_mma; c0 += 64) {              // two loads in flight per wait
+          uint32_t r0[32], r1[32];
+          tmem_ld32(t_addr + c0, r0);
+          tmem_ld32(t_addr + c0 + 32, r1);
+          tmem_wait_ld();
+          const int lim = A.n - (p * 256 + c0);
+          if (lim >= 64) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r0[j]));
+              bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r1[j]));
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (j < lim) bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r0[j]));
+              if (j + 32 < lim) bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r1[j]));
+            }
+          }
+        }
         for (; c0 + 32 <= n_mma; c0 += 32) {
           uint32_t r[32];
           tmem_ld32(t_addr + c0, r);
@@ -251,7 +271,7 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
           const int lim = A.n - (p * 256 + c0);
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (j < lim) best = fmaxf(best, __uint_as_float(r[j]));
+            if (j < lim) bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r[j]));
         }
         if (c0 < n_mma) {
           uint32_t r[16];
@@ -260,9 +280,10 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
           const int lim = A.n - (p * 256 + c0);
 #pragma unroll
           for (int j = 0; j < 16; ++j)
-            if (j < lim) best = fmaxf(best, __uint_as_float(r[j]));
+            if (j < lim) bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r[j]));
         }
       }
+      const float best = fmaxf(fmaxf(bacc[0], bacc[1]), fmaxf(bacc[2], bacc[3]));
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[slot]);
