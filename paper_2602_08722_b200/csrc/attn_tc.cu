@@ -25,7 +25,8 @@ namespace quoka {
 
 using namespace ptx;
 
-constexpr int kAttnThreads = 13 * 32;
+constexpr int kAttnThreads = 16 * 32;          // four warpgroups: softmax A, softmax B, loaders, MMA (+3 idle warps)
+constexpr int kRegsSoftmax = 184, kRegsOther = 72;   // (128-72)*256 registers move to the 256 softmax threads
 constexpr int kQTile = 128;
 constexpr int kKeyTile = 128;
 constexpr int kSlots = 5;
@@ -126,6 +127,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 
   if (warp < 8) {
     // ================================================================== softmax + epilogue
+    setmaxnreg_inc<kRegsSoftmax>();
     const int x = warp >> 2;                                  // Q tile A (0) or B (1)
     const int n_tiles = x ? g.n_b : g.n_a;
     const int quarter = warp & 3;
@@ -143,22 +145,22 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       tc_fence_after();
       const int lim = visible_cols<SPARSE>(g, j, row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
-      // ---- pass 1: row maximum of the raw logits
-      float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
+      // ---- the whole row of S in registers: one TMEM round trip per tile
+      uint32_t sr[128];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(s_addr + c * 32, r);
-        tmem_wait_ld();
-        if (masked) {
+      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr + c * 32);
+      tmem_wait_ld();
+      if (masked) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) if (c * 32 + i < lim) mxa[i & 3] = fmaxf(mxa[i & 3], __uint_as_float(r[i]));
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mxa[i & 3] = fmaxf(mxa[i & 3], __uint_as_float(r[i]));
-        }
+        for (int i = 0; i < 128; ++i) if (i >= lim) sr[i] = 0xFF800000u;      // -inf: exp2 gives exactly 0
       }
-      const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
+      float mxa[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mxa[i] = __uint_as_float(sr[i]);
+#pragma unroll
+      for (int i = 8; i < 128; ++i) mxa[i & 7] = fmaxf(mxa[i & 7], __uint_as_float(sr[i]));
+      const float mx = fmaxf(fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])),
+                             fmaxf(fmaxf(mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
       const float m_tile = mx * scale_log2;
       // ---- lazy rescale of the accumulator: only when some row's maximum grew by more than the threshold
       const bool grow = m_tile > m_run + kRescaleThreshold;
@@ -181,28 +183,18 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         m_run = m_new;
       }
       const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      // ---- pass 2: p = 2^(s*scale - m), row sum, bf16 P over the first 64 columns of S
+      // ---- p = 2^(s*scale - m), row sum, bf16 P over the first 64 columns of S
       float psa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(s_addr + c * 32, r);
-        tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), scale_log2, -m_use));
-          float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, -m_use));
-          if (masked) {
-            if (c * 32 + 2 * i >= lim) p0 = 0.f;
-            if (c * 32 + 2 * i + 1 >= lim) p1 = 0.f;
-          }
-          psa[i & 3] += p0 + p1;
-          const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-          pk[i] = *reinterpret_cast<const uint32_t*>(&b2);
-        }
-        tmem_st16(s_addr + c * 16, pk);
+      for (int i = 0; i < 64; ++i) {
+        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -m_use));
+        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -m_use));
+        psa[i & 3] += p0 + p1;
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+        sr[i] = *reinterpret_cast<const uint32_t*>(&b2);
       }
+      tmem_st32(s_addr, sr);
+      tmem_st32(s_addr + 32, sr + 32);
       l_run += (psa[0] + psa[1]) + (psa[2] + psa[3]);
       tmem_wait_st();
       tc_fence_before();
@@ -239,6 +231,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     }
   } else if (warp < 12) {
     // ================================================================== K / V row loaders (gather)
+    setmaxnreg_dec<kRegsOther>();
     const int lt = threadIdx.x - 8 * 32;                      // 0..127
     constexpr int PIECES = D / 8;                             // 16-byte pieces per row (16 or 8)
     constexpr int ROWS_PER_PASS = 128 / PIECES;               // rows the 128 loader threads cover at once
@@ -251,9 +244,9 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     int slot = 0, done_slot = 0;
     bool ok = true;
     const uint32_t kv_base = smem_u32(kv_smem);
-    // Element offset of each of this thread's rows of key tile j (-1 = past the end: zero fill).  The index
+    // Offset of each of this thread's rows of key tile j (all ones = past the end: zero fill).  The index
     // list and the page table are read here, one tile ahead of the copies that use them.
-    auto row_offsets = [&](int j, long long (&off)[RPT]) {
+    auto row_offsets = [&](int j, uint32_t (&off)[RPT]) {
       int t[RPT];
 #pragma unroll
       for (int i = 0; i < RPT; ++i) {
@@ -272,9 +265,10 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         }
       }
 #pragma unroll
-      for (int i = 0; i < RPT; ++i) off[i] = t[i] >= 0 ? kv_row_offset(P, s, kv, t[i]) + c16 * 8 : -1;
+      for (int i = 0; i < RPT; ++i)      // in 16-byte units; the host refuses caches beyond 2^32 of them
+        off[i] = t[i] >= 0 ? (uint32_t)(kv_row_offset(P, s, kv, t[i]) >> 3) + (uint32_t)c16 : 0xFFFFFFFFu;
     };
-    long long off_cur[RPT], off_next[RPT];
+    uint32_t off_cur[RPT], off_next[RPT];
     if (g.n_max > 0) row_offsets(0, off_cur);
     for (int it = 0; it < n_items; ++it) {
       if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) { ok = false; break; }
@@ -284,9 +278,9 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 #pragma unroll
       for (int i = 0; i < RPT; ++i) {
         const int rr = rsub + i * ROWS_PER_PASS;
-        const bool valid = off_cur[i] >= 0;
+        const bool valid = off_cur[i] != 0xFFFFFFFFu;
         const uint32_t dst = dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
-        cp_async_16(dst, valid ? src_base + off_cur[i] : src_base, valid);
+        cp_async_16(dst, reinterpret_cast<const uint4*>(src_base) + (valid ? off_cur[i] : 0u), valid);
       }
       cp_async_commit();
       if (!(it & 1)) {
@@ -314,7 +308,10 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         if (++done_slot == kSlots) done_slot = 0;
       }
     }
-  } else if (lane == 0) {
+  } else {
+    setmaxnreg_dec<kRegsOther>();
+  }
+  if (warp == 12 && lane == 0) {
     // ================================================================== MMA issuer (warp 12, one thread)
     mbar_arrive_expect_tx(q_full, 2 * kTileBytes);
     for (int x = 0; x < 2; ++x)
@@ -398,6 +395,9 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 // ---------------------------------------------------------------------------------------------- host
 bool attn_tc_supported(const quoka_params* p) {
   if (p->dtype != QUOKA_BF16) return false;
+  // the loaders address cache rows in 32-bit units of 16 bytes
+  const int64_t extent = (p->page_size ? p->kv_rows : (int64_t)p->batch) * p->kv_stride_b;
+  if (extent / 8 >= (int64_t)0xFFFFFFFFll) return false;
   return true;
 }
 
