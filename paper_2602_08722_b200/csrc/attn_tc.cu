@@ -30,7 +30,6 @@ constexpr int kRegsSoftmax = 184, kRegsOther = 72;   // (128-72)*256 registers m
 constexpr int kQTile = 128;
 constexpr int kKeyTile = 128;
 constexpr int kSlots = 5;
-constexpr int kLoaderLag = 3;               // key/value tiles in flight per loader thread
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
 bool encode_kv_tensor_map(CUtensorMap* out, const quoka_params* p, const void* cache, uint32_t box_rows);
@@ -95,26 +94,29 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
   unsigned char* q_smem = smem;                               // [2][HALVES][128][128 B]
   unsigned char* kv_smem = smem + 2 * kTileBytes;             // [kSlots][HALVES][128][128 B]
   uint64_t* bars = reinterpret_cast<uint64_t*>(kv_smem + (size_t)kSlots * kTileBytes);
-  uint64_t* kv_full = bars;                 // [kSlots]  4 loader warps arrive
+  uint64_t* kv_full = bars;                 // [kSlots]  128 loader threads' cp.async arrivals
   uint64_t* kv_empty = bars + kSlots;       // [kSlots]  MMA commit
   uint64_t* s_full = bars + 2 * kSlots;     // [2]       MMA commit
-  uint64_t* p_full = s_full + 2;            // [2]       4 softmax warps arrive
-  uint64_t* o_full = p_full + 2;            // [2]       MMA commit after the last PV
+  uint64_t* p_full = s_full + 2;            // [2][2]    4 softmax warps arrive, per Q tile and half of the key tile
+  uint64_t* o_full = p_full + 4;            // [2]       MMA commit after the last PV
   uint64_t* q_full = o_full + 2;            // TMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_full + 1);
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{&abort_flag, P.status};
-  const int s = blockIdx.z, h = blockIdx.y, kv = h / P.group;
-  const int rb = gridDim.x - 1 - blockIdx.x;                  // heaviest row blocks first
+  // grid = (heads, row blocks, batch): heads vary fastest so the CTAs resident together share a KV head's
+  // rows in L2, and the row blocks run heaviest (most causal tiles) first, lightest last
+  const int s = blockIdx.z, h = blockIdx.x, kv = h / P.group;
+  const int rb = gridDim.y - 1 - blockIdx.y;
   const int r0 = rb * 2 * kQTile;
   const AttnGeom g = make_geom<SPARSE>(P, s, r0, k_cnt);
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int i = 0; i < kSlots; ++i) { mbar_init(&kv_full[i], 4); mbar_init(&kv_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4); mbar_init(&o_full[i], 1); }
+    for (int i = 0; i < kSlots; ++i) { mbar_init(&kv_full[i], 128); mbar_init(&kv_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&o_full[i], 1); }
+    for (int i = 0; i < 4; ++i) mbar_init(&p_full[i], 4);
     mbar_init(q_full, 1);
     fence_mbar_init();
     tma_prefetch_desc(&tm_q);
@@ -183,23 +185,26 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         m_run = m_new;
       }
       const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      // ---- p = 2^(s*scale - m), row sum, bf16 P over the first 64 columns of S
+      // ---- p = 2^(s*scale - m), row sum; bf16 P is written over the first 64 columns of S
+      // and handed to the MMA issuer in two halves of 64 keys, so the first PV products run under the second half
       float psa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -m_use));
-        const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -m_use));
-        psa[i & 3] += p0 + p1;
-        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-        sr[i] = *reinterpret_cast<const uint32_t*>(&b2);
+      for (int half = 0; half < 2; ++half) {
+#pragma unroll
+        for (int i = half * 32; i < half * 32 + 32; ++i) {
+          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -m_use));
+          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -m_use));
+          psa[i & 3] += p0 + p1;
+          const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+          sr[i] = *reinterpret_cast<const uint32_t*>(&b2);
+        }
+        tmem_st32(s_addr + half * 32, sr + half * 32);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[2 * x + half]);
       }
-      tmem_st32(s_addr, sr);
-      tmem_st32(s_addr + 32, sr + 32);
       l_run += (psa[0] + psa[1]) + (psa[2] + psa[3]);
-      tmem_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&p_full[x]);
     }
     // ---- epilogue: O / l -> bf16 -> global
     if (ok && n_tiles > 0 && mbar_wait(&o_full[x], 0, wc)) {
@@ -241,8 +246,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     constexpr int RPT = kKeyTile / ROWS_PER_PASS;             // rows per thread per tile (16 or 8)
     const int n_items = 2 * g.n_max;
     uint32_t phase = 0;
-    int slot = 0, done_slot = 0;
-    bool ok = true;
+    int slot = 0;
     const uint32_t kv_base = smem_u32(kv_smem);
     // Offset of each of this thread's rows of key tile j (all ones = past the end: zero fill).  The index
     // list and the page table are read here, one tile ahead of the copies that use them.
@@ -271,7 +275,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     uint32_t off_cur[RPT], off_next[RPT];
     if (g.n_max > 0) row_offsets(0, off_cur);
     for (int it = 0; it < n_items; ++it) {
-      if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) { ok = false; break; }
+      if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) break;
       const int j = it >> 1;
       const __nv_bfloat16* src_base = (it & 1) ? vc : kc;
       const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
@@ -282,32 +286,18 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         const uint32_t dst = dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
         cp_async_16(dst, reinterpret_cast<const uint4*>(src_base) + (valid ? off_cur[i] : 0u), valid);
       }
-      cp_async_commit();
+      // this thread's share of the slot is signalled by the copy engine itself when the bytes have landed:
+      // no wait in the loader, every slot of the ring can be in flight
+      cp_async_mbar_arrive_noinc(&kv_full[slot]);
       if (!(it & 1)) {
         if (j + 1 < g.n_max) row_offsets(j + 1, off_next);    // in flight while the V copies are issued
       } else {
 #pragma unroll
         for (int i = 0; i < RPT; ++i) off_cur[i] = off_next[i];
       }
-      if (it >= kLoaderLag) {
-        cp_async_wait<kLoaderLag>();
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&kv_full[done_slot]);
-        if (++done_slot == kSlots) done_slot = 0;
-      }
       if (++slot == kSlots) { slot = 0; phase ^= 1; }
     }
-    cp_async_wait<0>();
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (ok) {
-      const int pending = n_items < kLoaderLag ? n_items : kLoaderLag;
-      for (int i = 0; i < pending; ++i) {
-        if (lane == 0) mbar_arrive(&kv_full[done_slot]);
-        if (++done_slot == kSlots) done_slot = 0;
-      }
-    }
+    cp_async_wait_all();                                      // nothing of this thread is in flight at exit
   } else {
     setmaxnreg_dec<kRegsOther>();
   }
@@ -327,6 +317,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     bool ok = mbar_wait(q_full, 0, wc);
     auto acquire = [&]() -> int {           // next ring item (K or V) becomes readable
       if (!mbar_wait(&kv_full[slot], kv_phase, wc)) { ok = false; return 0; }
+      fence_proxy_async_smem();             // cp.async wrote through the generic proxy, the MMA reads through the async one
       tc_fence_after();
       const int got = slot;
       if (++slot == kSlots) { slot = 0; kv_phase ^= 1; }
@@ -344,14 +335,17 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       mma_commit(&s_full[x]);
     };
     auto issue_pv = [&](int x, int vs, int j) {
-      if (!mbar_wait(&p_full[x], p_phase[x], wc)) { ok = false; return; }
-      p_phase[x] ^= 1;
-      tc_fence_after();
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {       // 16 keys per MMA: 8 packed columns of P, 16 rows of V
-        const uint64_t b = smem_desc_sw128(kv_base + vs * kTileBytes + kk * 2048, kHalfBytes, 1024);
-        mma_ts(tmem_base + O_COL[x], tmem_base + S_COL[x] + kk * 8, b, idesc_pv, (j | kk) ? 1u : 0u);
+      for (int half = 0; half < 2; ++half) {
+        if (!mbar_wait(&p_full[2 * x + half], p_phase[x], wc)) { ok = false; return; }
+        tc_fence_after();
+#pragma unroll
+        for (int kk = half * 4; kk < half * 4 + 4; ++kk) {   // 16 keys per MMA: 8 packed columns of P, 16 rows of V
+          const uint64_t b = smem_desc_sw128(kv_base + vs * kTileBytes + kk * 2048, kHalfBytes, 1024);
+          mma_ts(tmem_base + O_COL[x], tmem_base + S_COL[x] + kk * 8, b, idesc_pv, (j | kk) ? 1u : 0u);
+        }
       }
+      p_phase[x] ^= 1;
     };
     if (ok && g.n_max > 0) {
       k_slot = acquire();
@@ -413,7 +407,7 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
   const int halves = P.d / 64;
   const size_t tile = (size_t)halves * 128 * 128;
   const size_t smem = 1024 + (2 + kSlots) * tile + 512;
-  dim3 grid((P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.n_q, P.batch);
+  dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.batch);
   const bool sparse = k_idx != nullptr;
   cudaError_t e = cudaSuccess;
 #define QUOKA_ATTN_TC(H, S)                                                                                      \
