@@ -9,15 +9,18 @@
 //                    running max / sum in registers, P written back to tensor memory over S,
 //                    lazy rescale of the O accumulator (only when the max grew by more than 2^8),
 //                    final normalisation and the global store.
-//   warps 8-11       loaders: every K / V row of a tile is fetched with 16-byte cp.async straight
+//   warps 8-10       loaders: every K / V row of a tile is fetched with 16-byte cp.async straight
 //                    into the 128-byte-swizzled layout the MMA descriptors expect.  The row address
 //                    comes from the selected-index list (the gather), the chunk offset, or the page
 //                    table, so no compacted copy of K or V is ever made; rows past the end are
-//                    zero-filled.
-//   warp 12          MMA issuer (one thread): S = Q K^T (both operands in shared memory) and
+//                    zero-filled.  A slot's "full" barrier is armed by the copies themselves.
+//   warp 11          MMA issuer (one thread): S = Q K^T (both operands in shared memory) and
 //                    O += P V (P from tensor memory, V in shared memory, MN-major).
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, P aliasing the first 64 columns of its S.
 // K and V tiles share one ring of shared-memory slots in the order K0 V0 K1 V1 ...
+// 384 threads and no register re-balancing between roles: every thread may use 168 registers
+// (with 512 threads and setmaxnreg the compiler still scheduled the softmax for 128 registers,
+// which halved its speed).
 #include "sm100_ptx.cuh"
 #include "tensor_kernels.cuh"
 
@@ -25,8 +28,9 @@ namespace quoka {
 
 using namespace ptx;
 
-constexpr int kAttnThreads = 16 * 32;          // four warpgroups: softmax A, softmax B, loaders, MMA (+3 idle warps)
-constexpr int kRegsSoftmax = 184, kRegsOther = 72;   // (128-72)*256 registers move to the 256 softmax threads
+constexpr int kAttnThreads = 12 * 32;
+constexpr int kLoaderWarps = 3;
+constexpr int kMmaWarp = 11;
 constexpr int kQTile = 128;
 constexpr int kKeyTile = 128;
 constexpr int kSlots = 5;
@@ -80,6 +84,20 @@ __device__ __forceinline__ int visible_cols(const AttnGeom& g, int j, int row) {
   return max(0, min(kKeyTile, lim));
 }
 
+// Maximum of 32 score columns starting at col0; columns at and beyond `lim` are masked out.
+__device__ __forceinline__ float max32(uint32_t (&v)[32], bool masked, int col0, int lim) {
+  if (masked) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) if (col0 + i >= lim) v[i] = 0xFF800000u;    // -inf
+  }
+  float m[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) m[i] = __uint_as_float(v[i]);
+#pragma unroll
+  for (int i = 4; i < 32; ++i) m[i & 3] = fmaxf(m[i & 3], __uint_as_float(v[i]));
+  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+}
+
 template <int HALVES, bool SPARSE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv_bfloat16* __restrict__ kc,
@@ -94,7 +112,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
   unsigned char* q_smem = smem;                               // [2][HALVES][128][128 B]
   unsigned char* kv_smem = smem + 2 * kTileBytes;             // [kSlots][HALVES][128][128 B]
   uint64_t* bars = reinterpret_cast<uint64_t*>(kv_smem + (size_t)kSlots * kTileBytes);
-  uint64_t* kv_full = bars;                 // [kSlots]  128 loader threads' cp.async arrivals
+  uint64_t* kv_full = bars;                 // [kSlots]  the loader threads' cp.async arrivals
   uint64_t* kv_empty = bars + kSlots;       // [kSlots]  MMA commit
   uint64_t* s_full = bars + 2 * kSlots;     // [2]       MMA commit
   uint64_t* p_full = s_full + 2;            // [2][2]    4 softmax warps arrive, per Q tile and half of the key tile
@@ -114,14 +132,14 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int i = 0; i < kSlots; ++i) { mbar_init(&kv_full[i], 128); mbar_init(&kv_empty[i], 1); }
+    for (int i = 0; i < kSlots; ++i) { mbar_init(&kv_full[i], kLoaderWarps * 32); mbar_init(&kv_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&o_full[i], 1); }
     for (int i = 0; i < 4; ++i) mbar_init(&p_full[i], 4);
     mbar_init(q_full, 1);
     fence_mbar_init();
     tma_prefetch_desc(&tm_q);
   }
-  if (warp == 12) tmem_alloc(tmem_slot, 512);
+  if (warp == kMmaWarp) tmem_alloc(tmem_slot, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -129,7 +147,6 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 
   if (warp < 8) {
     // ================================================================== softmax + epilogue
-    setmaxnreg_inc<kRegsSoftmax>();
     const int x = warp >> 2;                                  // Q tile A (0) or B (1)
     const int n_tiles = x ? g.n_b : g.n_a;
     const int quarter = warp & 3;
@@ -147,22 +164,25 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       tc_fence_after();
       const int lim = visible_cols<SPARSE>(g, j, row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
-      // ---- the whole row of S in registers: one TMEM round trip per tile
-      uint32_t sr[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr + c * 32);
-      tmem_wait_ld();
-      if (masked) {
-#pragma unroll
-        for (int i = 0; i < 128; ++i) if (i >= lim) sr[i] = 0xFF800000u;      // -inf: exp2 gives exactly 0
+      // ---- pass 1: the row maximum, 32 columns at a time with the next load in flight.  The row is read
+      // once here and once more by pass 2: tensor memory is cheap to re-read, and not keeping 128 values
+      // live leaves pass 2 the registers it needs to keep a whole block of exponentials in flight.
+      float mx;
+      {
+        uint32_t c0[32], c1[32];
+        tmem_ld32(s_addr, c0);
+        tmem_wait_ld();
+        tmem_ld32(s_addr + 32, c1);
+        mx = max32(c0, masked, 0, lim);
+        tmem_wait_ld();
+        tmem_ld32(s_addr + 64, c0);
+        mx = fmaxf(mx, max32(c1, masked, 32, lim));
+        tmem_wait_ld();
+        tmem_ld32(s_addr + 96, c1);
+        mx = fmaxf(mx, max32(c0, masked, 64, lim));
+        tmem_wait_ld();
+        mx = fmaxf(mx, max32(c1, masked, 96, lim));
       }
-      float mxa[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) mxa[i] = __uint_as_float(sr[i]);
-#pragma unroll
-      for (int i = 8; i < 128; ++i) mxa[i & 7] = fmaxf(mxa[i & 7], __uint_as_float(sr[i]));
-      const float mx = fmaxf(fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])),
-                             fmaxf(fmaxf(mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
       const float m_tile = mx * scale_log2;
       // ---- lazy rescale of the accumulator: only when some row's maximum grew by more than the threshold
       const bool grow = m_tile > m_run + kRescaleThreshold;
@@ -185,20 +205,29 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         m_run = m_new;
       }
       const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      // ---- p = 2^(s*scale - m), row sum; bf16 P is written over the first 64 columns of S
-      // and handed to the MMA issuer in two halves of 64 keys, so the first PV products run under the second half
+      // ---- pass 2: p = 2^(s*scale - m) in two blocks of 64 keys.  bf16 P goes over the first 64 columns of
+      // S (block h of P lands on columns 32h..32h+31, all of them read already) and each block is handed to the
+      // MMA issuer as soon as it is stored, so the first PV products run under the second block's arithmetic.
       float psa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
+        uint32_t v[64], pk[32];
+        tmem_ld32(s_addr + half * 64, v);
+        tmem_ld32(s_addr + half * 64 + 32, v + 32);
+        tmem_wait_ld();
+        if (masked) {
 #pragma unroll
-        for (int i = half * 32; i < half * 32 + 32; ++i) {
-          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), scale_log2, -m_use));
-          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), scale_log2, -m_use));
+          for (int i = 0; i < 64; ++i) if (half * 64 + i >= lim) v[i] = 0xFF800000u;   // -inf: exp2 gives exactly 0
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), scale_log2, -m_use));
+          const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), scale_log2, -m_use));
           psa[i & 3] += p0 + p1;
           const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-          sr[i] = *reinterpret_cast<const uint32_t*>(&b2);
+          pk[i] = *reinterpret_cast<const uint32_t*>(&b2);
         }
-        tmem_st32(s_addr + half * 32, sr + half * 32);
+        tmem_st32(s_addr + half * 32, pk);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -234,43 +263,62 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       if (store && lse)
         lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
     }
-  } else if (warp < 12) {
+  } else if (warp < 8 + kLoaderWarps) {
     // ================================================================== K / V row loaders (gather)
-    setmaxnreg_dec<kRegsOther>();
-    const int lt = threadIdx.x - 8 * 32;                      // 0..127
+    // One warp instruction copies 32 / PIECES whole rows (16 lanes x 16 bytes cover a 256-byte row); the
+    // row groups of a tile are dealt round-robin to the loader warps.
+    const int lw = warp - 8;
     constexpr int PIECES = D / 8;                             // 16-byte pieces per row (16 or 8)
-    constexpr int ROWS_PER_PASS = 128 / PIECES;               // rows the 128 loader threads cover at once
-    const int c16 = lt % PIECES;                              // this thread's piece of the row
-    const int rsub = lt / PIECES;
+    constexpr int ROWS_PER_INSTR = 32 / PIECES;               // 2 or 4
+    constexpr int GROUPS = kKeyTile / ROWS_PER_INSTR;         // 64 or 32 row groups per tile
+    constexpr int RPT = (GROUPS + kLoaderWarps - 1) / kLoaderWarps;   // row groups per warp (last one may be idle)
+    const int c16 = lane % PIECES;                            // this thread's piece of the row
+    const int rsub = lane / PIECES;
     const int32_t* idx = SPARSE ? k_idx + ((long long)s * P.n_kv + kv) * P.budget_cap : nullptr;
-    constexpr int RPT = kKeyTile / ROWS_PER_PASS;             // rows per thread per tile (16 or 8)
     const int n_items = 2 * g.n_max;
     uint32_t phase = 0;
     int slot = 0;
     const uint32_t kv_base = smem_u32(kv_smem);
+    // Row addressing in 16-byte units, 32 bits wide (the host refuses caches beyond 2^32 units; strides are
+    // multiples of 8 elements): sequence/head base plus this thread's piece, row stride, page stride.
+    const uint32_t st16 = (uint32_t)(P.kv_st >> 3), sb16 = (uint32_t)(P.kv_sb >> 3);
+    const uint32_t base16 = (uint32_t)(((P.page_size == 0 ? (long long)s * P.kv_sb : 0ll) + (long long)kv * P.kv_sh) >> 3) +
+                            (uint32_t)c16;
     // Offset of each of this thread's rows of key tile j (all ones = past the end: zero fill).  The index
     // list and the page table are read here, one tile ahead of the copies that use them.
     auto row_offsets = [&](int j, uint32_t (&off)[RPT]) {
       int t[RPT];
 #pragma unroll
       for (int i = 0; i < RPT; ++i) {
-        const int rr = rsub + i * ROWS_PER_PASS;
-        if (SPARSE) {
-          if (j < g.n_sel) {
-            const int u = j * kKeyTile + rr;
-            t[i] = u < g.cnt ? __ldg(idx + u) : -1;
+        const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
+        t[i] = -1;
+        if (rr < kKeyTile) {
+          if (SPARSE) {
+            if (j < g.n_sel) {
+              const int u = j * kKeyTile + rr;
+              if (u < g.cnt) t[i] = __ldg(idx + u);
+            } else {
+              const int pos = (j - g.n_sel) * kKeyTile + rr;
+              if (pos < P.chunk) t[i] = g.T + pos;
+            }
           } else {
-            const int pos = (j - g.n_sel) * kKeyTile + rr;
-            t[i] = pos < P.chunk ? g.T + pos : -1;
+            const int tt = j * kKeyTile + rr;
+            if (tt < g.T + P.chunk) t[i] = tt;
           }
-        } else {
-          const int tt = j * kKeyTile + rr;
-          t[i] = tt < g.T + P.chunk ? tt : -1;
         }
       }
 #pragma unroll
-      for (int i = 0; i < RPT; ++i)      // in 16-byte units; the host refuses caches beyond 2^32 of them
-        off[i] = t[i] >= 0 ? (uint32_t)(kv_row_offset(P, s, kv, t[i]) >> 3) + (uint32_t)c16 : 0xFFFFFFFFu;
+      for (int i = 0; i < RPT; ++i) {
+        uint32_t o = 0xFFFFFFFFu;
+        if (t[i] >= 0) {
+          if (P.page_size == 0) o = base16 + (uint32_t)t[i] * st16;
+          else {
+            const uint32_t page = (uint32_t)__ldg(P.block_table + (long long)s * P.max_pages + (t[i] >> 6));
+            o = page * sb16 + base16 + (uint32_t)(t[i] & (kPage - 1)) * st16;
+          }
+        }
+        off[i] = o;
+      }
     };
     uint32_t off_cur[RPT], off_next[RPT];
     if (g.n_max > 0) row_offsets(0, off_cur);
@@ -281,10 +329,12 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
 #pragma unroll
       for (int i = 0; i < RPT; ++i) {
-        const int rr = rsub + i * ROWS_PER_PASS;
-        const bool valid = off_cur[i] != 0xFFFFFFFFu;
-        const uint32_t dst = dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
-        cp_async_16(dst, reinterpret_cast<const uint4*>(src_base) + (valid ? off_cur[i] : 0u), valid);
+        const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
+        if (rr < kKeyTile) {
+          const bool valid = off_cur[i] != 0xFFFFFFFFu;
+          const uint32_t dst = dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
+          cp_async_16(dst, reinterpret_cast<const uint4*>(src_base) + (valid ? off_cur[i] : 0u), valid);
+        }
       }
       // this thread's share of the slot is signalled by the copy engine itself when the bytes have landed:
       // no wait in the loader, every slot of the ring can be in flight
@@ -298,11 +348,8 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       if (++slot == kSlots) { slot = 0; phase ^= 1; }
     }
     cp_async_wait_all();                                      // nothing of this thread is in flight at exit
-  } else {
-    setmaxnreg_dec<kRegsOther>();
-  }
-  if (warp == 12 && lane == 0) {
-    // ================================================================== MMA issuer (warp 12, one thread)
+  } else if (lane == 0) {
+    // ================================================================== MMA issuer (one thread)
     mbar_arrive_expect_tx(q_full, 2 * kTileBytes);
     for (int x = 0; x < 2; ++x)
       for (int hh = 0; hh < HALVES; ++hh)
@@ -355,19 +402,16 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         mma_commit(&kv_empty[k_slot]);
       }
       for (int j = 0; ok && j < g.n_max; ++j) {
-        v_slot = acquire();
-        if (!ok) break;
         const bool more = j + 1 < g.n_max;
+        v_slot = acquire();
+        if (ok && more) k_slot = acquire();     // both are normally there already: keeps the waits off the P -> PV -> QK chain
+        if (!ok) break;
         if (j < g.n_a) {
           issue_pv(0, v_slot, j);
           if (!ok) break;
           if (j + 1 == g.n_a) mma_commit(&o_full[0]);
         }
-        if (more) {
-          k_slot = acquire();
-          if (!ok) break;
-          if (j + 1 < g.n_a) issue_qk(0, k_slot);
-        }
+        if (more && j + 1 < g.n_a) issue_qk(0, k_slot);
         if (j < g.n_b) {
           issue_pv(1, v_slot, j);
           if (!ok) break;
@@ -383,7 +427,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 12) tmem_dealloc(tmem_base, 512);
+  if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
 // ---------------------------------------------------------------------------------------------- host
