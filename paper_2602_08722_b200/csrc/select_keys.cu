@@ -1,20 +1,20 @@
 // Top-B key selection (Algorithm 1: I = topk(S^, B_SA)) as a radix select.
 //
-// One CTA per (sequence, KV head).  The fp32 scores are mapped to order-preserving uint32 codes;
-// four 8-bit passes, most significant digit first, narrow a (prefix, need) pair until `prefix` is the
-// code of the B-th largest score and `need` is how many rows with exactly that code are still to be
-// taken.  Digit histograms live in shared memory and are filled with warp-aggregated atomics
-// (match + popc, one atomic per distinct digit per warp); the bin holding the B-th largest is found
-// by one warp with a shuffle prefix sum.  The output pass walks the rows in position order and
-// computes each selected row's slot with warp ballots and a block prefix sum, so the list comes out
+// The fp32 scores are mapped to order-preserving uint32 codes; digit passes, most significant first,
+// narrow a (prefix, need) pair until `prefix` is the code of the B-th largest score and `need` is how
+// many rows with exactly that code are still to be taken.  The output pass walks the rows in position
+// order and computes each selected row's slot with warp ballots and prefix sums, so the list comes out
 // ascending and rows that tie at the threshold are taken lowest position first.
 //
-// Two kernels share that scheme.  select_keys_cluster_kernel (the default) gives each (sequence, KV
-// head) a thread-block cluster of 8 CTAs: every CTA keeps its contiguous slice of the row in shared
-// memory as order codes (one read of the scores from HBM, all later passes on chip), the per-CTA
-// digit histograms are summed through distributed shared memory, and the per-CTA selected counts are
-// prefix-summed the same way so the output stays ascending across the cluster.  select_keys_kernel
-// (one CTA per head, scores re-read from L2 every pass) serves rows too long for the slices.
+// select_keys_reg_kernel (the default): one CTA of 1024 threads per (sequence, KV head), or a cluster
+// of 2/4/8 CTAs for long rows, holds the whole row as order codes IN REGISTERS (up to 32 per thread:
+// the scores are read from memory exactly once, coalesced).  Three passes of 12 + 12 + 8 bits: each
+// pass histograms only the rows still matching the prefix with shared-memory atomics (a warp whose
+// lanes all carry the same digit adds once), the bin holding the B-th largest is found with a block-wide
+// suffix scan, and with a cluster the per-CTA histograms and counts are summed through distributed
+// shared memory.
+// select_keys_kernel (one CTA per head, scores re-read from L2 every pass, 8-bit digits) serves rows
+// too long for that.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -126,51 +126,24 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_kernel(DevParams P, c
   }
 }
 
-constexpr int kSelCluster = 8;
-constexpr int kSelMaxSlice = 53248;       // order codes per CTA that fit in shared memory (208 KiB)
 
-// Finds, among 256 bins summed over the cluster, the bin in which the running count (from bin 255
-// down) reaches `need`.  Called by warp 0; lane l owns bins 255-8l .. 248-8l.
-__device__ __forceinline__ void find_bin(const uint32_t* tot, uint32_t need, uint32_t prefix, int shift, int lane,
-                                         uint32_t* s_prefix, uint32_t* s_need) {
-  uint32_t c[8], sum = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) { c[i] = tot[255 - 8 * lane - i]; sum += c[i]; }
-  uint32_t incl = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  const uint32_t hit = __ballot_sync(0xFFFFFFFFu, incl >= need);
-  if (lane == (__ffs(hit) - 1)) {
-    uint32_t cum = incl - sum;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (cum + c[i] >= need) {
-        *s_prefix = prefix | ((uint32_t)(255 - 8 * lane - i) << shift);
-        *s_need = need - cum;
-        break;
-      }
-      cum += c[i];
-    }
-  }
-}
+constexpr int kRegBins = 4096;            // 12-bit digits
+constexpr int kHistWords = 2 * kRegBins + 256;
 
-__global__ void __launch_bounds__(kSelThreads) select_keys_cluster_kernel(DevParams P, const float* __restrict__ scores,
-                                                                           int32_t* __restrict__ k_idx,
-                                                                           int32_t* __restrict__ k_cnt) {
-  extern __shared__ uint32_t keys[];            // this CTA's slice as order codes
-  __shared__ uint32_t hist[256];
-  __shared__ uint32_t tot[256];
+// Warp w of CTA r owns positions [r*1024*ITEMS + w*32*ITEMS, +32*ITEMS); lane l holds i*32 + l of them.
+template <int ITEMS, int CL>
+__global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams P, const float* __restrict__ scores,
+                                                                       int32_t* __restrict__ k_idx,
+                                                                       int32_t* __restrict__ k_cnt) {
+  __shared__ uint32_t hist_all[kHistWords];     // one histogram per pass, zeroed once: no barrier to re-use one
   __shared__ uint32_t s_prefix, s_need;
-  __shared__ uint32_t my_cnt[2];                // rows of my slice above / equal to the threshold
-  __shared__ uint32_t warp_tot[32];
+  __shared__ uint32_t warp_val[32];
   __shared__ uint32_t warp_off[33];
+  __shared__ uint32_t cta_cnt[2];               // rows of this CTA above / equal to the threshold
 
   cg::cluster_group cluster = cg::this_cluster();
-  const int rank = (int)cluster.block_rank();
-  const int head = blockIdx.x / kSelCluster;
+  const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
+  const int head = blockIdx.x / CL;
   const int s = head / P.n_kv, kv = head % P.n_kv;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int T = __ldg(P.ctx_len + s);
@@ -178,137 +151,180 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_cluster_kernel(DevPar
   const float* row = scores + (long long)head * P.max_ctx;
   int32_t* out = k_idx + (long long)head * P.budget_cap;
   const int gtid = rank * kSelThreads + tid;
-  constexpr int kAll = kSelCluster * kSelThreads;
+  constexpr int kAll = CL * kSelThreads;
   if (kv == 0 && gtid == 0) k_cnt[s] = B;
   for (int i = B + gtid; i < P.budget_cap; i += kAll) out[i] = -1;
   if (B <= 0) return;                           // uniform over the cluster
-  if (B >= T) {
+  if (B >= T) {                                 // budget covers the cache: identity
     for (int i = gtid; i < T; i += kAll) out[i] = i;
     return;
   }
-  // slice [lo, hi) of the row, a multiple of the block size so the output pass sees whole chunks
-  const int slice = ((T + kSelCluster - 1) / kSelCluster + kSelThreads - 1) / kSelThreads * kSelThreads;
-  const int lo = min(T, rank * slice), hi = min(T, lo + slice);
-  const int n = hi - lo;
-  for (int i0 = 0; i0 < n; i0 += 4 * kSelThreads) {      // four independent loads in flight per thread
-    float v[4];
+  const int base = (rank * kSelThreads + wid * 32) * ITEMS + lane;      // position of item i: base + 32 i
+  uint32_t code[ITEMS];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = i0 + u * kSelThreads + tid;
-      v[u] = i < n ? __ldg(row + lo + i) : 0.f;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = i0 + u * kSelThreads + tid;
-      if (i < n) keys[i] = float_order_key(v[u]);
-    }
+  for (int i = 0; i < ITEMS; ++i) {
+    const int pos = base + 32 * i;
+    code[i] = pos < T ? float_order_key(__ldg(row + pos)) : 0u;
   }
-  uint32_t prefix = 0, mask = 0, need = (uint32_t)B;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();                            // also orders the slice stores before the first pass
-    for (int i0 = 0; i0 < n; i0 += kSelThreads) {
-      const int i = i0 + tid;
-      const bool in = i < n;
-      const uint32_t key = in ? keys[i] : 0u;
-      const bool live = in && ((key & mask) == prefix);
-      const uint32_t digit = live ? ((key >> shift) & 255u) : 256u + (uint32_t)lane;
-      const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-      if (live && lane == (__ffs(peers) - 1)) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
-    }
-    cluster.sync();                             // every CTA's histogram is complete
-    if (tid < 256) {
-      uint32_t sum = 0;
-#pragma unroll
-      for (int r = 0; r < kSelCluster; ++r) sum += cluster.map_shared_rank(hist, r)[tid];
-      tot[tid] = sum;
-    }
-    __syncthreads();
-    if (wid == 0) find_bin(tot, need, prefix, shift, lane, &s_prefix, &s_need);
-    cluster.sync();                             // peers are done reading my histogram before it is zeroed
-    prefix = s_prefix;
-    need = s_need;
-    mask |= 255u << shift;
-  }
-  const uint32_t thr = prefix;
-  // rows of my slice above / equal to the threshold, then the offsets of my slice in the output
-  uint32_t c_gt = 0, c_eq = 0;
-  for (int i = tid; i < n; i += kSelThreads) {
-    const uint32_t key = keys[i];
-    c_gt += key > thr;
-    c_eq += key == thr;
-  }
-  c_gt = __reduce_add_sync(0xFFFFFFFFu, c_gt);
-  c_eq = __reduce_add_sync(0xFFFFFFFFu, c_eq);
-  if (tid < 2) my_cnt[tid] = 0;
+  for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
   __syncthreads();
-  if (lane == 0) { atomicAdd(&my_cnt[0], c_gt); atomicAdd(&my_cnt[1], c_eq); }
-  cluster.sync();
-  uint32_t run_gt = 0, run_eq = 0;
-  for (int r = 0; r < rank; ++r) {
-    const uint32_t* pc = cluster.map_shared_rank(my_cnt, r);
-    run_gt += pc[0];
-    run_eq += pc[1];
-  }
-  for (int i0 = 0; i0 < n; i0 += kSelThreads) {
-    const int i = i0 + tid;
-    const uint32_t key = (i < n) ? keys[i] : 0u;
-    const bool gt = (i < n) && key > thr;
-    const bool eq = (i < n) && key == thr;
-    const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt);
-    const uint32_t b_eq = __ballot_sync(0xFFFFFFFFu, eq);
-    if (lane == 0) warp_tot[wid] = (uint32_t)__popc(b_gt) | ((uint32_t)__popc(b_eq) << 16);
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t prefix = 0, mask = 0, need = (uint32_t)B;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
+    const int nb = pass == 2 ? 256 : kRegBins;
+    uint32_t* hist = hist_all + pass * kRegBins;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+      const bool live = (base + 32 * i < T) && ((code[i] & mask) == prefix);
+      if (live) atomicAdd(&hist[(code[i] >> shift) & (uint32_t)(nb - 1)], 1u);
+    }
+    if (CL > 1) cluster.sync(); else __syncthreads();
+    // thread t owns the 4 bins nb-1-4t .. nb-4-4t (descending); find where the running count reaches `need`
+    uint32_t c[4] = {0, 0, 0, 0}, sum = 0;
+    if (4 * tid < nb) {
+      if (CL > 1) {
+#pragma unroll
+        for (int r = 0; r < CL; ++r) {              // independent remote loads, all in flight together
+          const uint32_t* ph = cluster.map_shared_rank(hist, r);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) c[k] += ph[nb - 1 - (4 * tid + k)];
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) c[k] = hist[nb - 1 - (4 * tid + k)];
+      }
+      sum = (c[0] + c[1]) + (c[2] + c[3]);
+    }
+    uint32_t incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_val[wid] = incl;
     __syncthreads();
     if (wid == 0) {
-      const uint32_t v = warp_tot[lane];
-      uint32_t incl = v;
+      const uint32_t v = warp_val[lane];
+      uint32_t w = v;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += u;
+        const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, w, o);
+        if (lane >= o) w += u;
       }
-      warp_off[lane] = incl - v;
-      if (lane == 31) warp_off[32] = incl;
+      warp_off[lane] = w - v;
     }
     __syncthreads();
-    const uint32_t off = warp_off[wid], total = warp_off[32];
-    const uint32_t lt = (1u << lane) - 1u;
-    const uint32_t gt_before = run_gt + (off & 0xFFFFu) + (uint32_t)__popc(b_gt & lt);
-    const uint32_t eq_before = run_eq + (off >> 16) + (uint32_t)__popc(b_eq & lt);
-    if (gt || (eq && eq_before < need)) out[gt_before + min(eq_before, need)] = lo + i;
-    run_gt += total & 0xFFFFu;
-    run_eq += total >> 16;
+    const uint32_t excl = warp_off[wid] + incl - sum;
+    if (excl < need && need <= excl + sum) {          // exactly one thread
+      uint32_t cum = excl;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (cum + c[k] >= need) {
+          s_prefix = prefix | ((uint32_t)(nb - 1 - (4 * tid + k)) << shift);
+          s_need = need - cum;
+          break;
+        }
+        cum += c[k];
+      }
+    }
+    __syncthreads();
+    prefix = s_prefix;
+    need = s_need;
+    mask |= (uint32_t)(nb - 1) << shift;
   }
-  cluster.sync();                               // my_cnt stays mapped until every peer has read it
+  // prefix = code of the B-th largest score; take every row above it and the first `need` rows equal to it
+  const uint32_t thr = prefix;
+  uint32_t w_gt = 0, w_eq = 0;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const bool in = base + 32 * i < T;
+    w_gt += (in && code[i] > thr) ? 1u : 0u;
+    w_eq += (in && code[i] == thr) ? 1u : 0u;
+  }
+  w_gt = __reduce_add_sync(0xFFFFFFFFu, w_gt);
+  w_eq = __reduce_add_sync(0xFFFFFFFFu, w_eq);
+  if (lane == 0) warp_val[wid] = w_gt | (w_eq << 16);      // at most 1024 each
+  __syncthreads();
+  if (wid == 0) {
+    const uint32_t v = warp_val[lane];
+    uint32_t g = v & 0xFFFFu, e = v >> 16, gi = g, ei = e;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t ug = __shfl_up_sync(0xFFFFFFFFu, gi, o), ue = __shfl_up_sync(0xFFFFFFFFu, ei, o);
+      if (lane >= o) { gi += ug; ei += ue; }
+    }
+    warp_off[lane] = gi - g;                 // exclusive counts of rows above the threshold ...
+    warp_val[lane] = ei - e;                 // ... and equal to it, over the warps before this one
+    if (lane == 31) { cta_cnt[0] = gi; cta_cnt[1] = ei; }
+  }
+  if (CL > 1) cluster.sync(); else __syncthreads();
+  uint32_t run_gt = warp_off[wid], run_eq = warp_val[wid];
+  if (CL > 1) {
+    uint32_t pg[CL], pe[CL];
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {               // independent remote loads
+      const uint32_t* pc = cluster.map_shared_rank(cta_cnt, r);
+      pg[r] = pc[0];
+      pe[r] = pc[1];
+    }
+#pragma unroll
+    for (int r = 0; r < CL; ++r)
+      if (r < rank) { run_gt += pg[r]; run_eq += pe[r]; }
+  }
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const int pos = base + 32 * i;
+    const bool in = pos < T;
+    const bool gt = in && code[i] > thr, eq = in && code[i] == thr;
+    const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt), b_eq = __ballot_sync(0xFFFFFFFFu, eq);
+    const uint32_t gt_before = run_gt + (uint32_t)__popc(b_gt & lt);
+    const uint32_t eq_before = run_eq + (uint32_t)__popc(b_eq & lt);
+    if (gt || (eq && eq_before < need)) out[gt_before + min(eq_before, need)] = pos;
+    run_gt += (uint32_t)__popc(b_gt);
+    run_eq += (uint32_t)__popc(b_eq);
+  }
+  if (CL > 1) cluster.sync();                   // histograms and counts stay mapped until every peer has read them
+}
+
+template <int ITEMS, int CL>
+static cudaError_t launch_reg(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt, cudaStream_t st) {
+  if (CL == 1) {
+    select_keys_reg_kernel<ITEMS, CL><<<P.batch * P.n_kv, kSelThreads, 0, st>>>(P, scores, k_idx, k_cnt);
+    return cudaSuccess;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(P.batch * P.n_kv * CL);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CL;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_keys_reg_kernel<ITEMS, CL>, P, scores, k_idx, k_cnt);
 }
 
 cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt,
                                cudaStream_t st) {
-  const int slice = ((P.max_ctx + kSelCluster - 1) / kSelCluster + kSelThreads - 1) / kSelThreads * kSelThreads;
-  if (slice <= kSelMaxSlice) {
-    const size_t smem = (size_t)(slice > 0 ? slice : 1) * sizeof(uint32_t);
-    cudaError_t e = cudaFuncSetAttribute(select_keys_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(P.batch * P.n_kv * kSelCluster);
-    cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kSelCluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, select_keys_cluster_kernel, P, scores, k_idx, k_cnt);
-    count_launch();
-    return e != cudaSuccess ? e : cudaGetLastError();
-  }
-  select_keys_kernel<<<P.batch * P.n_kv, kSelThreads, 0, st>>>(P, scores, k_idx, k_cnt);
+  // One CTA per head while the row fits its registers (32 per thread); clusters only for longer rows: merging
+  // the histograms through distributed shared memory costs more than it saves on a short row.
+  const int per_thread = (P.max_ctx + kSelThreads - 1) / kSelThreads;    // items per thread with one CTA per head
+  cudaError_t e;
+  if (per_thread <= 4) e = launch_reg<4, 1>(P, scores, k_idx, k_cnt, st);
+  else if (per_thread <= 8) e = launch_reg<8, 1>(P, scores, k_idx, k_cnt, st);
+  else if (per_thread <= 16) e = launch_reg<16, 1>(P, scores, k_idx, k_cnt, st);
+  else if (per_thread <= 32) e = launch_reg<32, 1>(P, scores, k_idx, k_cnt, st);
+  else if (per_thread <= 64) e = launch_reg<32, 2>(P, scores, k_idx, k_cnt, st);
+  else if (per_thread <= 128) e = launch_reg<32, 4>(P, scores, k_idx, k_cnt, st);
+  else if (per_thread <= 256) e = launch_reg<32, 8>(P, scores, k_idx, k_cnt, st);
+  else { select_keys_kernel<<<P.batch * P.n_kv, kSelThreads, 0, st>>>(P, scores, k_idx, k_cnt); e = cudaSuccess; }
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace quoka

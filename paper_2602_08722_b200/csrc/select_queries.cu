@@ -1,60 +1,139 @@
 // Query sub-selection, normalisation and GQA pre-aggregation (Algorithm 1, first two blocks).
 //
-// rank_queries : one CTA per (sequence, query head).  Pass 1 sums the head's C query rows into the
-//                mean query M; pass 2 computes CosSim(q_r, M) for every row (the second read of
-//                the head's rows hits L2); a shared-memory bitonic sort of (cosine, position)
-//                codes yields the N lowest cosines in ascending order, equal cosines by position.
+// rank_queries : a thread-block cluster of 8 CTAs per (sequence, query head); each CTA owns a
+//                contiguous slice of the head's C query rows.  Pass 1 reads the slice from HBM once
+//                (16-byte vector loads, D/8 lanes per row), keeps it in shared memory, and sums it
+//                into the CTA's share of the mean query; the shares are added across the cluster
+//                through distributed shared memory in a fixed order.  Pass 2 computes
+//                CosSim(q_r, M) for every row of the slice from shared memory, sorts the slice's
+//                (cosine, position) codes with a shared-memory bitonic sort, and places each of its
+//                N smallest by global rank: own rank + binary searches in the seven peers' sorted
+//                slices.  Codes are unique (the position is part of them), so the N lowest cosines
+//                come out in ascending order, equal cosines by position.
 // aggregate    : one warp per (sequence, KV head, rank j): mean over the G heads of the group of
 //                their j-th retained query, each divided by its own norm; one rounding to dtype.
-// Both are HBM/L2-bound passes over Q: rows are read with 16-byte vector loads, D/8 lanes per row.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace quoka {
 
-constexpr int kRankThreads = 1024;
+constexpr int kRankThreads = 512;
+constexpr int kRankCluster = 8;
+constexpr size_t kRankStageLimit = 160 * 1024;   // a slice larger than this is re-read from L2 in pass 2
+
+template <typename T> struct Raw8;                // 8 consecutive elements as 16-byte words
+template <> struct Raw8<__nv_bfloat16> { uint4 w[1]; };
+template <> struct Raw8<float> { uint4 w[2]; };
+
+template <typename T>
+__device__ __forceinline__ void raw_to_f32(const Raw8<T>& r, float (&x)[8]) {
+  if constexpr (sizeof(T) == 2) {
+    const uint32_t w[4] = {r.w[0].x, r.w[0].y, r.w[0].z, r.w[0].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      x[2 * j] = __uint_as_float(w[j] << 16);
+      x[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    }
+  } else {
+    x[0] = __uint_as_float(r.w[0].x); x[1] = __uint_as_float(r.w[0].y);
+    x[2] = __uint_as_float(r.w[0].z); x[3] = __uint_as_float(r.w[0].w);
+    x[4] = __uint_as_float(r.w[1].x); x[5] = __uint_as_float(r.w[1].y);
+    x[6] = __uint_as_float(r.w[1].z); x[7] = __uint_as_float(r.w[1].w);
+  }
+}
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P, const T* __restrict__ q,
-                                                                     int32_t* __restrict__ q_idx) {
+                                                                     int32_t* __restrict__ q_idx, int rpc, int n_sort,
+                                                                     int staged, int m_peer) {
   constexpr int LG = D / 8;                 // lanes per row, 8 elements each
   constexpr int RPI = kRankThreads / LG;    // rows per iteration
+  constexpr int NW = sizeof(T) * 8 / 16;    // 16-byte words per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  // dynamic shared memory: sort keys | reduction buffer | row norms | staged rows
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);               // [n_sort]
+  float* red = reinterpret_cast<float*>(smem_raw + (size_t)n_sort * 8);                     // [RPI][D]
+  float* norms = red + RPI * D;                                                             // [rpc]
+  unsigned long long* peer_keys = reinterpret_cast<unsigned long long*>(norms + ((rpc + 3) & ~3));   // [7][m_peer]
+  uint4* rows = reinterpret_cast<uint4*>(peer_keys + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1));   // [rpc][LG][NW]
+  __shared__ float part[D];                 // this CTA's share of the column sums
   __shared__ float M[D];
   __shared__ float Mnorm;
 
-  const int s = blockIdx.x / P.n_q;
-  const int h = blockIdx.x % P.n_q;
-  const int C = P.chunk;
-  const int N = P.n_sel;
-  int32_t* out = q_idx + ((int64_t)s * P.n_q + h) * N;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int head = blockIdx.x / kRankCluster;
+  const int s = head / P.n_q, h = head % P.n_q;
+  const int C = P.chunk, N = P.n_sel;
+  int32_t* out = q_idx + (long long)head * N;
   const int tid = threadIdx.x;
 
   if (C <= P.n_retain) {                    // no sub-selection: every query, in position order
-    for (int j = tid; j < C; j += kRankThreads) out[j] = j;
+    for (int j = rank * kRankThreads + tid; j < C; j += kRankCluster * kRankThreads) out[j] = j;
     return;
   }
 
-  const T* qh = q + (int64_t)s * P.q_sb + (int64_t)h * P.q_sh;
+  const T* qh = q + (long long)s * P.q_sb + (long long)h * P.q_sh;
   const int lane_in_row = tid % LG;
   const int row_slot = tid / LG;
+  const int lo = min(C, rank * rpc), hi = min(C, lo + rpc);
+  const int n_loc = hi - lo;
 
-  // ---- pass 1: column sums -> mean query
+  // ---- pass 1: the slice goes to shared memory with every 16-byte copy in flight at once (one HBM round
+  // trip for the whole slice), then column sums and row norms are taken from there
+  if (staged) {
+    constexpr int WPR = LG * NW;                             // 16-byte words per row
+    constexpr int EPW = 16 / (int)sizeof(T);                 // elements per word
+    const uint32_t rows_s = (uint32_t)__cvta_generic_to_shared(rows);
+    for (int w = tid; w < n_loc * WPR; w += kRankThreads) {
+      const int r = w / WPR, c = w % WPR;
+      const T* src = qh + (long long)(lo + r) * P.q_st + c * EPW;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(rows_s + (uint32_t)w * 16u), "l"(src) : "memory");
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncthreads();
+  }
   float acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-  for (int r = row_slot; r < C; r += RPI) {
-    float x[8];
-    load_vec<T, 8>(qh + (int64_t)r * P.q_st + lane_in_row * 8, x);
+  for (int r0 = 0; r0 < n_loc; r0 += RPI) {                // uniform trip count: the shuffles below need whole warps
+    const int r = r0 + row_slot;
+    float nn = 0.f;
+    if (r < n_loc) {
+      Raw8<T> raw;
+      if (staged) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] += x[i];
+        for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)r * LG + lane_in_row) * NW + w];
+      } else {
+        const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)(lo + r) * P.q_st + lane_in_row * 8);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) raw.w[w] = __ldg(src + w);
+      }
+      float x[8];
+      raw_to_f32<T>(raw, x);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { acc[i] += x[i]; nn = fmaf(x[i], x[i], nn); }
+    }
+#pragma unroll
+    for (int o = LG / 2; o > 0; o >>= 1) nn += __shfl_xor_sync(0xFFFFFFFFu, nn, o);
+    if (lane_in_row == 0 && r < n_loc) norms[r] = fmaxf(sqrtf(nn), kNormEps);
   }
-  float* red = reinterpret_cast<float*>(smem_raw);        // [RPI][D]
 #pragma unroll
   for (int i = 0; i < 8; ++i) red[row_slot * D + lane_in_row * 8 + i] = acc[i];
   __syncthreads();
   if (tid < D) {
     float sum = 0.f;
     for (int r = 0; r < RPI; ++r) sum += red[r * D + tid];
+    part[tid] = sum;
+  }
+  cluster.sync();
+  if (tid < D) {
+    float sum = 0.f;
+#pragma unroll
+    for (int r = 0; r < kRankCluster; ++r) sum += cluster.map_shared_rank(part, r)[tid];   // fixed order
     M[tid] = sum / (float)C;
   }
   __syncthreads();
@@ -64,42 +143,45 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
     p = warp_sum(p);
     if (tid == 0) Mnorm = fmaxf(sqrtf(p), kNormEps);
   }
-  __syncthreads();   // also: everyone is done reading `red` before the sort buffer overwrites it
+  __syncthreads();
 
-  // ---- pass 2: cosine of every row to M, packed as (order code << 32 | position)
-  int n_sort = 1;
-  while (n_sort < C) n_sort <<= 1;
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
+  // ---- pass 2: cosine of every row of the slice to M, packed as (order code << 32 | position)
   float m[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) m[i] = M[lane_in_row * 8 + i];
   const float mn = Mnorm;
   for (int r0 = 0; r0 < n_sort; r0 += RPI) {
     const int r = r0 + row_slot;
-    float dot = 0.f, nn = 0.f;
-    if (r < C) {
+    float dot = 0.f;
+    if (r < n_loc) {
+      Raw8<T> raw;
+      if (staged) {
+#pragma unroll
+        for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)r * LG + lane_in_row) * NW + w];
+      } else {
+        const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)(lo + r) * P.q_st + lane_in_row * 8);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) raw.w[w] = __ldg(src + w);
+      }
       float x[8];
-      load_vec<T, 8>(qh + (int64_t)r * P.q_st + lane_in_row * 8, x);
+      raw_to_f32<T>(raw, x);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { dot += x[i] * m[i]; nn += x[i] * x[i]; }
+      for (int i = 0; i < 8; ++i) dot = fmaf(x[i], m[i], dot);
     }
 #pragma unroll
-    for (int o = LG / 2; o > 0; o >>= 1) {
-      dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
-      nn += __shfl_xor_sync(0xFFFFFFFFu, nn, o);
-    }
+    for (int o = LG / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
     if (lane_in_row == 0 && r < n_sort) {
       unsigned long long code = ~0ull;                    // padding sorts last
-      if (r < C) {
-        const float c = dot / (fmaxf(sqrtf(nn), kNormEps) * mn);
-        code = ((unsigned long long)float_order_key(c) << 32) | (unsigned)r;
+      if (r < n_loc) {
+        const float c = dot / (norms[r] * mn);
+        code = ((unsigned long long)float_order_key(c) << 32) | (unsigned)(lo + r);
       }
       keys[r] = code;
     }
   }
   __syncthreads();
 
-  // ---- bitonic sort, ascending
+  // ---- bitonic sort of the slice, ascending
   for (int k = 2; k <= n_sort; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
       for (int i = tid; i < n_sort; i += kRankThreads) {
@@ -113,7 +195,34 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
       __syncthreads();
     }
   }
-  for (int j = tid; j < N; j += kRankThreads) out[j] = (int32_t)(keys[j] & 0xFFFFFFFFull);
+  cluster.sync();                                         // every slice is sorted
+
+  // ---- global rank of my N smallest: own rank + number of smaller codes in each peer's slice.  Only a
+  // peer's first m_peer = min(n_sort, N) codes matter (more smaller ones than that already push the rank past
+  // N); they are copied into local shared memory first, because a chain of dependent remote reads is slow.
+  for (int e = tid; e < (kRankCluster - 1) * m_peer; e += kRankThreads) {
+    const int pr = e / m_peer, j = e % m_peer;
+    const int r = pr + (pr >= rank ? 1 : 0);
+    peer_keys[e] = cluster.map_shared_rank(keys, r)[j];
+  }
+  __syncthreads();
+  const int n_cand = min(N, n_loc);
+  for (int li = tid; li < n_cand; li += kRankThreads) {
+    const unsigned long long key = keys[li];
+    int rk = li;
+#pragma unroll 1
+    for (int pr = 0; pr < kRankCluster - 1; ++pr) {
+      const unsigned long long* pk = peer_keys + (size_t)pr * m_peer;
+      int a = 0, b = m_peer;                              // first index with pk[idx] >= key
+      while (a < b) {
+        const int mid = (a + b) >> 1;
+        if (pk[mid] < key) a = mid + 1; else b = mid;
+      }
+      rk += a;
+    }
+    if (rk < N) out[rk] = (int32_t)(key & 0xFFFFFFFFull);
+  }
+  cluster.sync();                                         // my keys stay mapped until every peer is done
 }
 
 template <typename T, int D>
@@ -132,18 +241,38 @@ __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, con
   float acc[NE];
 #pragma unroll
   for (int i = 0; i < NE; ++i) acc[i] = 0.f;
-  for (int g = 0; g < P.group; ++g) {
-    const int h = kv * P.group + g;
-    const int r = __ldg(q_idx + ((int64_t)s * P.n_q + h) * N + j);
-    float x[NE];
-    load_vec<T, NE>(q + (int64_t)s * P.q_sb + (int64_t)h * P.q_sh + (int64_t)r * P.q_st + lane * NE, x);
-    float nn = 0.f;
+  for (int g0 = 0; g0 < P.group; g0 += 32) {
+    // the group's ranks in one load, then the rows four at a time so their loads overlap
+    const int gl = g0 + lane;
+    const int r_lane = gl < P.group ? __ldg(q_idx + ((int64_t)s * P.n_q + kv * P.group + gl) * N + j) : 0;
+    const int g_end = min(32, P.group - g0);
+    for (int g4 = 0; g4 < g_end; g4 += 4) {
+      float x[4][NE];
 #pragma unroll
-    for (int i = 0; i < NE; ++i) nn += x[i] * x[i];
-    nn = warp_sum(nn);
-    const float norm = fmaxf(sqrtf(nn), kNormEps);
+      for (int u = 0; u < 4; ++u) {
+        const int g = g4 + u;
+        const int r = __shfl_sync(0xFFFFFFFFu, r_lane, g & 31);
+        if (g < g_end) {
+          const int h = kv * P.group + g0 + g;
+          load_vec<T, NE>(q + (int64_t)s * P.q_sb + (int64_t)h * P.q_sh + (int64_t)r * P.q_st + lane * NE, x[u]);
+        } else {
 #pragma unroll
-    for (int i = 0; i < NE; ++i) acc[i] += x[i] / norm;
+          for (int i = 0; i < NE; ++i) x[u][i] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float nn = 0.f;
+#pragma unroll
+        for (int i = 0; i < NE; ++i) nn += x[u][i] * x[u][i];
+        nn = warp_sum(nn);
+        const float norm = fmaxf(sqrtf(nn), kNormEps);
+        if (g4 + u < g_end) {
+#pragma unroll
+          for (int i = 0; i < NE; ++i) acc[i] += x[u][i] / norm;
+        }
+      }
+    }
   }
   const float inv_g = 1.f / (float)P.group;
 #pragma unroll
@@ -151,27 +280,40 @@ __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, con
   store_vec<T, NE>(qbar + warp * D + lane * NE, acc);
 }
 
+template <typename T, int D>
+static cudaError_t launch_rank_t(const DevParams& P, const void* q, int32_t* q_idx, cudaStream_t st) {
+  constexpr int LG = D / 8, RPI = kRankThreads / LG;
+  int rpc = (P.chunk + kRankCluster - 1) / kRankCluster;
+  int n_sort = 2;
+  while (n_sort < rpc) n_sort <<= 1;
+  const size_t row_bytes = (size_t)rpc * D * sizeof(T);
+  const int m_peer = n_sort < P.n_sel ? n_sort : P.n_sel;
+  const size_t fixed = (size_t)n_sort * 8 + (size_t)RPI * D * 4 + (size_t)((rpc + 3) & ~3) * 4 + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1) * 8;
+  const int staged = fixed + row_bytes <= kRankStageLimit + 48 * 1024 && row_bytes <= kRankStageLimit ? 1 : 0;
+  const size_t smem = fixed + (staged ? row_bytes : 0);
+  cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(P.batch * P.n_q * kRankCluster);
+  cfg.blockDim = dim3(kRankThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kRankCluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, rank_queries_kernel<T, D>, P, (const T*)q, q_idx, rpc, n_sort, staged, m_peer);
+}
+
 cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st) {
-  int n_sort = 1;
-  while (n_sort < P.chunk) n_sort <<= 1;
-  size_t smem = (size_t)n_sort * 8;
-  if (smem < 32768) smem = 32768;           // the pass-1 reduction buffer [RPI][D] floats is 32 KiB
-  const int grid = P.batch * P.n_q;
-#define QUOKA_RANK(T, D)                                                                                       \
-  do {                                                                                                         \
-    cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                         (int)smem);                                                           \
-    if (e != cudaSuccess) return e;                                                                            \
-    rank_queries_kernel<T, D><<<grid, kRankThreads, smem, st>>>(P, (const T*)q, q_idx);                         \
-  } while (0)
-  if (dtype == QUOKA_BF16) {
-    if (P.d == 128) QUOKA_RANK(__nv_bfloat16, 128); else QUOKA_RANK(__nv_bfloat16, 64);
-  } else {
-    if (P.d == 128) QUOKA_RANK(float, 128); else QUOKA_RANK(float, 64);
-  }
-#undef QUOKA_RANK
+  cudaError_t e;
+  if (dtype == QUOKA_BF16) e = P.d == 128 ? launch_rank_t<__nv_bfloat16, 128>(P, q, q_idx, st) : launch_rank_t<__nv_bfloat16, 64>(P, q, q_idx, st);
+  else e = P.d == 128 ? launch_rank_t<float, 128>(P, q, q_idx, st) : launch_rank_t<float, 64>(P, q, q_idx, st);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, const int32_t* q_idx, void* qbar,
