@@ -75,7 +75,8 @@ def sum_work(w, ctx_lens):
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples every 200 ms while the timed region runs."""
+    """SM clock and throttle-reason samples taken while the timed region runs: NVML every 5 ms in a thread
+    (read-only queries), or nvidia-smi every 200 ms when NVML is not importable."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -84,8 +85,24 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines = []
+        self.samples = []
+        self.stop_flag = False
+        self.nvml = None
+        self.th = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = int(vis.split(",")[self.index]) if vis and vis.split(",")[self.index].isdigit() else self.index
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.nvml = pynvml
+            self.th = threading.Thread(target=self._poll, daemon=True)
+            self.th.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "200"],
@@ -95,20 +112,42 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        while not self.stop_flag:
+            try:
+                sm = n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)
+                mx = n.nvmlDeviceGetMaxClockInfo(self.handle, n.NVML_CLOCK_SM)
+                rs = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle) if hasattr(n, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                self.samples.append((sm, mx, rs))
+            except Exception:
+                pass
+            time.sleep(0.005)
+
     def _pump(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
     def stop(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.th.join(timeout=2)
+            bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
+            reasons = sorted(k for k, b in bits.items() if any(r & b for _, _, r in self.samples))
+            sm = [x[0] for x in self.samples]
+            mx = [x[1] for x in self.samples]
+            return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                    "samples": len(sm), "source": "nvml 5 ms", "reasons": reasons}
         if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["no clock source available"]}
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
@@ -122,7 +161,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "source": "nvidia-smi 200 ms", "reasons": sorted(reasons)}
 
 
 # ----------------------------------------------------------------------------- timing helpers
@@ -192,7 +231,7 @@ def host_threads():
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama8b_32k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -217,7 +256,8 @@ def main():
               "head_dim": w["d"], "ctx_len": w["T"] if w["T"] is not None else ctx_lens, "chunk_len": w["C"],
               "n_retain": w["n_retain"], "kv_budget": w.get("kv_budget", 0), "budget_frac": w.get("budget_frac", 0.0),
               "paged": bool(w.get("paged")), "parallelism": f"independent chunks x{world}",
-              "l2": "flushed between timed steps (512 MiB write outside the event pairs)"}
+              "l2": "flushed between timed steps (512 MiB write outside the event pairs)",
+              "kernel_timing": "stages back to back on one stream, CUDA events between them, L2 flushed before each sequence"}
 
     if args.impl == "reference":
         if rank != 0:
@@ -317,7 +357,9 @@ def main():
                               "note": "fused-only run (profiling aid); not a bench line"}))
         return 0
 
-    # ---- per-kernel timings through the staged entry points (each alone, L2 flushed between launches)
+    # ---- per-kernel timings: the staged entry points run back to back on the stream, exactly as the fused call
+    # issues them, with a CUDA event between stages (a kernel timed alone after an idle stream carries ~10 us of
+    # launch latency, which hides the small kernels); L2 is flushed before each sequence
     ksteps = max(5, min(args.steps, 20))
     stages = {
         "select_queries": lambda: api.quoka_select_queries(p, q, q_idx, qbar, ws),
@@ -327,9 +369,21 @@ def main():
     }
     work = sum_work(w, ctx_lens)
     pk = peaks()
+    samples = {name: [] for name in stages}
+    for it in range(ksteps + 3):
+        flush()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)]
+        evs[0].record()
+        for i, fn in enumerate(stages.values()):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            for i, name in enumerate(stages):
+                samples[name].append(evs[i].elapsed_time(evs[i + 1]) * 1e3)
     kernels = {}
-    for name, fn in stages.items():
-        ts = time_loop(fn, ksteps, 3, flush)
+    for name in stages:
+        ts = samples[name]
         us = statistics.mean(ts)
         kernels[name] = {"us": round(us, 2), "min_us": round(min(ts), 2),
                          "gbs": round(work[name]["bytes"] / us / 1e3, 1),
