@@ -44,6 +44,15 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Packed pairs of fp32 (one instruction for two lanes of arithmetic) and the three-input maximum: the softmax
+// threads share their sub-partition's issue port with the loaders and the MMA issuer, so instructions count.
+__device__ __forceinline__ uint64_t pack2(float a, float b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ uint64_t pack2u(uint32_t a, uint32_t b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b)); return r; }
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+
 struct AttnGeom {
   int T, cnt, n_sel;        // cached length, selected rows, selected tiles (sparse); cnt = T, n_sel unused (dense)
   int n_a, n_b, n_max;      // key tiles Q tile A / B take part in, and their maximum
@@ -90,12 +99,13 @@ __device__ __forceinline__ float max32(uint32_t (&v)[32], bool masked, int col0,
 #pragma unroll
     for (int i = 0; i < 32; ++i) if (col0 + i >= lim) v[i] = 0xFF800000u;    // -inf
   }
-  float m[4];
+  float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) m[i] = __uint_as_float(v[i]);
-#pragma unroll
-  for (int i = 4; i < 32; ++i) m[i & 3] = fmaxf(m[i & 3], __uint_as_float(v[i]));
-  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+  for (int i = 2; i < 30; i += 4) {
+    m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+    m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+  }
+  return max3(m0, m1, fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31])));
 }
 
 template <int HALVES, bool SPARSE>
@@ -208,7 +218,8 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       // ---- pass 2: p = 2^(s*scale - m) in two blocks of 64 keys.  bf16 P goes over the first 64 columns of
       // S (block h of P lands on columns 32h..32h+31, all of them read already) and each block is handed to the
       // MMA issuer as soon as it is stored, so the first PV products run under the second block's arithmetic.
-      float psa[4] = {0.f, 0.f, 0.f, 0.f};
+      const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m_use, -m_use);
+      uint64_t psa[2] = {0ull, 0ull};                           // four running sums as two packed pairs
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t v[64], pk[32];
@@ -221,9 +232,10 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         }
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), scale_log2, -m_use));
-          const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), scale_log2, -m_use));
-          psa[i & 3] += p0 + p1;
+          float x0, x1;
+          unpack2(fma2(pack2u(v[2 * i], v[2 * i + 1]), sc2, nm2), x0, x1);
+          const float p0 = ex2(x0), p1 = ex2(x1);
+          psa[i & 1] = add2(psa[i & 1], pack2(p0, p1));
           const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
           pk[i] = *reinterpret_cast<const uint32_t*>(&b2);
         }
@@ -233,7 +245,10 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_full[2 * x + half]);
       }
-      l_run += (psa[0] + psa[1]) + (psa[2] + psa[3]);
+      float ps0, ps1, ps2, ps3;
+      unpack2(psa[0], ps0, ps1);
+      unpack2(psa[1], ps2, ps3);
+      l_run += (ps0 + ps1) + (ps2 + ps3);
     }
     // ---- epilogue: O / l -> bf16 -> global
     if (ok && n_tiles > 0 && mbar_wait(&o_full[x], 0, wc)) {
