@@ -299,67 +299,67 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     const uint32_t st16 = (uint32_t)(P.kv_st >> 3), sb16 = (uint32_t)(P.kv_sb >> 3);
     const uint32_t base16 = (uint32_t)(((P.page_size == 0 ? (long long)s * P.kv_sb : 0ll) + (long long)kv * P.kv_sh) >> 3) +
                             (uint32_t)c16;
-    // Offset of each of this thread's rows of key tile j (all ones = past the end: zero fill).  The index
-    // list and the page table are read here, one tile ahead of the copies that use them.
-    auto row_offsets = [&](int j, uint32_t (&off)[RPT]) {
-      int t[RPT];
+    const int32_t* table = P.block_table + (long long)s * P.max_pages;
+    // Row numbers of this thread's rows of a tile of the selected list (-1 past the end).  They are fetched one
+    // tile ahead and only looked at when that tile's copies are issued, so the loader never waits on them.
+    // The per-row code below is kept free of branches (clamped loads, selects): a branch per row costs a single
+    // warp far more than the arithmetic it skips.
+    auto list_rows = [&](int j, int (&t)[RPT]) {
+      if (SPARSE && j < g.n_sel) {
+        const int last = g.cnt - 1 - j * kKeyTile;                 // last valid row of this tile (>= 0)
 #pragma unroll
-      for (int i = 0; i < RPT; ++i) {
-        const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
-        t[i] = -1;
-        if (rr < kKeyTile) {
-          if (SPARSE) {
-            if (j < g.n_sel) {
-              const int u = j * kKeyTile + rr;
-              if (u < g.cnt) t[i] = __ldg(idx + u);
-            } else {
-              const int pos = (j - g.n_sel) * kKeyTile + rr;
-              if (pos < P.chunk) t[i] = g.T + pos;
-            }
-          } else {
-            const int tt = j * kKeyTile + rr;
-            if (tt < g.T + P.chunk) t[i] = tt;
-          }
+        for (int i = 0; i < RPT; ++i) {
+          const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
+          const int v = __ldg(idx + j * kKeyTile + min(rr, last));
+          t[i] = rr <= last ? v : -1;
         }
-      }
-#pragma unroll
-      for (int i = 0; i < RPT; ++i) {
-        uint32_t o = 0xFFFFFFFFu;
-        if (t[i] >= 0) {
-          if (P.page_size == 0) o = base16 + (uint32_t)t[i] * st16;
-          else {
-            const uint32_t page = (uint32_t)__ldg(P.block_table + (long long)s * P.max_pages + (t[i] >> 6));
-            o = page * sb16 + base16 + (uint32_t)(t[i] & (kPage - 1)) * st16;
-          }
-        }
-        off[i] = o;
       }
     };
-    uint32_t off_cur[RPT], off_next[RPT];
-    if (g.n_max > 0) row_offsets(0, off_cur);
+    int t_cur[RPT], t_next[RPT];
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) t_next[i] = -1;
+    list_rows(0, t_next);
     for (int it = 0; it < n_items; ++it) {
       if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) break;
       const int j = it >> 1;
-      const __nv_bfloat16* src_base = (it & 1) ? vc : kc;
+      const bool from_list = SPARSE && j < g.n_sel;
+      if (!(it & 1)) {
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) t_cur[i] = t_next[i];
+      }
+      // rows outside the list are consecutive: row_first + r for r < row_count (the chunk's own rows, or all rows)
+      int row_first, row_count;
+      if (SPARSE) { row_first = g.T + (j - g.n_sel) * kKeyTile; row_count = P.chunk - (j - g.n_sel) * kKeyTile; }
+      else { row_first = j * kKeyTile; row_count = g.T + P.chunk - j * kKeyTile; }
+      const uint4* src_base = reinterpret_cast<const uint4*>((it & 1) ? vc : kc);
       const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
+      int t[RPT];                                                 // row number, or -1
 #pragma unroll
       for (int i = 0; i < RPT; ++i) {
         const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
-        if (rr < kKeyTile) {
-          const bool valid = off_cur[i] != 0xFFFFFFFFu;
-          const uint32_t dst = dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4);
-          cp_async_16(dst, reinterpret_cast<const uint4*>(src_base) + (valid ? off_cur[i] : 0u), valid);
+        t[i] = from_list ? t_cur[i] : (rr < row_count ? row_first + rr : -1);
+      }
+      uint32_t off[RPT];
+      if (P.page_size == 0) {
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) off[i] = base16 + (uint32_t)max(t[i], 0) * st16;
+      } else {
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) {
+          const int tc = max(t[i], 0);
+          off[i] = (uint32_t)__ldg(table + (tc >> 6)) * sb16 + base16 + (uint32_t)(tc & (kPage - 1)) * st16;
         }
+      }
+#pragma unroll
+      for (int i = 0; i < RPT; ++i) {
+        const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
+        if (rr < kKeyTile)                                        // false only for the last group of some warps
+          cp_async_16(dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4), src_base + off[i], t[i] >= 0);
       }
       // this thread's share of the slot is signalled by the copy engine itself when the bytes have landed:
       // no wait in the loader, every slot of the ring can be in flight
       cp_async_mbar_arrive_noinc(&kv_full[slot]);
-      if (!(it & 1)) {
-        if (j + 1 < g.n_max) row_offsets(j + 1, off_next);    // in flight while the V copies are issued
-      } else {
-#pragma unroll
-        for (int i = 0; i < RPT; ++i) off_cur[i] = off_next[i];
-      }
+      if (!(it & 1)) list_rows(j + 1, t_next);
       if (++slot == kSlots) { slot = 0; phase ^= 1; }
     }
     cp_async_wait_all();                                      // nothing of this thread is in flight at exit
