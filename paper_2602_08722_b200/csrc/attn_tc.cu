@@ -385,26 +385,34 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       if (++slot == kSlots) { slot = 0; kv_phase ^= 1; }
       return got;
     };
+    // Operand descriptors are built once; a tile, slot or k-step offset is an addition to the 16-byte-unit
+    // address field (shared memory addresses stay far below the field's 14 bits), which keeps the issuing
+    // thread's instruction count per MMA small.
+    const uint64_t desc_q = smem_desc_sw128(q_base, 16, 1024);
+    const uint64_t desc_k = smem_desc_sw128(kv_base, 16, 1024);            // K-major rows (K tiles)
+    const uint64_t desc_v = smem_desc_sw128(kv_base, kHalfBytes, 1024);    // MN-major rows (V tiles)
     auto issue_qk = [&](int x, int ks) {
+      const uint64_t da = desc_q + (uint64_t)(x * (kTileBytes >> 4));
+      const uint64_t db = desc_k + (uint64_t)((uint32_t)ks * (kTileBytes >> 4));
 #pragma unroll
       for (int hh = 0; hh < HALVES; ++hh)
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
-          const uint64_t a = smem_desc_sw128(q_base + x * kTileBytes + hh * kHalfBytes + kk * 32, 16, 1024);
-          const uint64_t b = smem_desc_sw128(kv_base + ks * kTileBytes + hh * kHalfBytes + kk * 32, 16, 1024);
-          mma_ss(tmem_base + S_COL[x], a, b, idesc_qk, (hh | kk) ? 1u : 0u);
+          const uint64_t off = (uint64_t)((hh * kHalfBytes + kk * 32) >> 4);
+          mma_ss(tmem_base + S_COL[x], da + off, db + off, idesc_qk, (hh | kk) ? 1u : 0u);
         }
       mma_commit(&s_full[x]);
     };
     auto issue_pv = [&](int x, int vs, int j) {
+      const uint64_t dv = desc_v + (uint64_t)((uint32_t)vs * (kTileBytes >> 4));
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         if (!mbar_wait(&p_full[2 * x + half], p_phase[x], wc)) { ok = false; return; }
         tc_fence_after();
 #pragma unroll
         for (int kk = half * 4; kk < half * 4 + 4; ++kk) {   // 16 keys per MMA: 8 packed columns of P, 16 rows of V
-          const uint64_t b = smem_desc_sw128(kv_base + vs * kTileBytes + kk * 2048, kHalfBytes, 1024);
-          mma_ts(tmem_base + O_COL[x], tmem_base + S_COL[x] + kk * 8, b, idesc_pv, (j | kk) ? 1u : 0u);
+          mma_ts(tmem_base + O_COL[x], tmem_base + S_COL[x] + kk * 8, dv + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
+                 (j | kk) ? 1u : 0u);
         }
       }
       p_phase[x] ^= 1;

@@ -164,7 +164,8 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
     const int pos = base + 32 * i;
-    code[i] = pos < T ? float_order_key(__ldg(row + pos)) : 0u;
+    const uint32_t c = float_order_key(__ldg(row + min(pos, T - 1)));      // clamped load, no branch per item
+    code[i] = pos < T ? c : 0u;
   }
   for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
   __syncthreads();
