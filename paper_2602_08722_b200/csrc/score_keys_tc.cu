@@ -24,7 +24,7 @@ namespace quoka {
 using namespace ptx;
 
 constexpr int kTileKeys = 128;
-constexpr int kScoreThreads = 192;          // 6 warps
+constexpr int kScoreThreads = 320;          // 10 warps: TMA, MMA, two epilogue groups of four
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxStages = 8;
 
@@ -210,12 +210,24 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue: 4 warps, one key per thread
+    // ------------------------------------------------------------------ epilogue: one key per thread.
+    // Two groups of four warps take alternate tiles (group g = accumulator slot g), because one tile's epilogue
+    // (key norm from shared memory, 128 accumulator columns from tensor memory) takes longer than the tile's
+    // share of HBM time.  With a single accumulator slot (N > 256) only group 0 works.
+    const int group = (warp - 2) >> 2;
     const int quarter = warp & 3;                       // TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;                // key row within the tile
     TileWalk w; w.seek(P, lo, hi);
     int stage = 0; uint32_t phase = 0; int slot = 0; uint32_t acc_phase = 0;
-    for (; w.valid(); w.next(P)) {
+    int n_done = 0;                                     // tiles walked so far
+    for (; w.valid(); w.next(P), ++n_done) {
+      const bool mine = slots == 2 ? ((n_done & 1) == group) : (group == 0);
+      if (!mine) {                                      // the other group's tile: only keep the ring position
+        if (++stage == A.stages) { stage = 0; phase ^= 1; }
+        continue;
+      }
+      slot = slots == 2 ? group : 0;
+      acc_phase = slots == 2 ? (uint32_t)((n_done >> 1) & 1) : (uint32_t)(n_done & 1);
       if (!mbar_wait(&full[stage], phase, wc)) break;
       // |k|^2 from the tile in shared memory (rotated 16-byte reads: conflict-free)
       float nacc[4] = {0.f, 0.f, 0.f, 0.f};                 // independent partial sums: no 256-deep FMA chain
@@ -252,10 +264,7 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
           const int lim = A.n - (p * 256 + c0);
           if (lim >= 64) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r0[j]));
-              bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r1[j]));
-            }
+            for (int j = 0; j < 32; ++j) bacc[j & 3] = max3(bacc[j & 3], __uint_as_float(r0[j]), __uint_as_float(r1[j]));
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -291,7 +300,6 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
       if (t < __ldg(P.ctx_len + w.s))
         scores[((long long)w.s * P.n_kv + w.kv) * P.max_ctx + t] = best / fmaxf(sqrtf(nn), kNormEps);
       if (++stage == A.stages) { stage = 0; phase ^= 1; }
-      if (++slot == slots) { slot = 0; acc_phase ^= 1; }
     }
   }
   tc_fence_before();
