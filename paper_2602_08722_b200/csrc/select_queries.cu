@@ -54,8 +54,9 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   constexpr int NW = sizeof(T) * 8 / 16;    // 16-byte words per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // dynamic shared memory: sort keys | reduction buffer | row norms | staged rows
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);               // [n_sort]
-  float* red = reinterpret_cast<float*>(smem_raw + (size_t)n_sort * 8);                     // [RPI][D]
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);               // [n_sort] 32-key sorted runs
+  unsigned long long* sorted = keys + n_sort;                                               // [n_sort] the sorted slice
+  float* red = reinterpret_cast<float*>(smem_raw + (size_t)n_sort * 16);                    // [RPI][D]
   float* norms = red + RPI * D;                                                             // [rpc]
   unsigned long long* peer_keys = reinterpret_cast<unsigned long long*>(norms + ((rpc + 3) & ~3));   // [7][m_peer]
   uint4* rows = reinterpret_cast<uint4*>(peer_keys + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1));   // [rpc][LG][NW]
@@ -82,44 +83,67 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   const int lo = min(C, rank * rpc), hi = min(C, lo + rpc);
   const int n_loc = hi - lo;
 
-  // ---- pass 1: the slice goes to shared memory with every 16-byte copy in flight at once (one HBM round
-  // trip for the whole slice), then column sums and row norms are taken from there
+  // ---- pass 1: the slice goes to shared memory with every 16-byte copy in flight at once, committed in 8
+  // groups of rows; column sums and row norms are taken group by group as the copies land, so the arithmetic
+  // runs under the HBM transfer
+  const int n_iter = (n_loc + RPI - 1) / RPI;                // 32/64-row trips over the slice
+  const int grp_rows = ((n_iter + 7) / 8) * RPI;             // rows per copy group
   if (staged) {
     constexpr int WPR = LG * NW;                             // 16-byte words per row
     constexpr int EPW = 16 / (int)sizeof(T);                 // elements per word
     const uint32_t rows_s = (uint32_t)__cvta_generic_to_shared(rows);
-    for (int w = tid; w < n_loc * WPR; w += kRankThreads) {
-      const int r = w / WPR, c = w % WPR;
-      const T* src = qh + (long long)(lo + r) * P.q_st + c * EPW;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(rows_s + (uint32_t)w * 16u), "l"(src) : "memory");
+#pragma unroll 1
+    for (int gi = 0; gi < 8; ++gi) {
+      const int w_lo = min(n_loc, gi * grp_rows) * WPR, w_hi = min(n_loc, (gi + 1) * grp_rows) * WPR;
+      for (int w = w_lo + tid; w < w_hi; w += kRankThreads) {
+        const int r = w / WPR, c = w % WPR;
+        const T* src = qh + (long long)(lo + r) * P.q_st + c * EPW;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(rows_s + (uint32_t)w * 16u), "l"(src) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    __syncthreads();
   }
   float acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-  for (int r0 = 0; r0 < n_loc; r0 += RPI) {                // uniform trip count: the shuffles below need whole warps
-    const int r = r0 + row_slot;
-    float nn = 0.f;
-    if (r < n_loc) {
+#pragma unroll
+  for (int gi = 0; gi < 8; ++gi) {
+    if (staged) {
+      switch (gi) {                                          // all but the 7 - gi newest groups have landed
+        case 0: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+      }
+      __syncthreads();
+    }
+    const int g_lo = min(n_loc, gi * grp_rows), g_hi = min(n_loc, (gi + 1) * grp_rows);
+    for (int r0 = g_lo; r0 < g_hi; r0 += RPI) {              // uniform trip count: the shuffles below need whole warps
+      const int r = r0 + row_slot;
+      float nn = 0.f;
       Raw8<T> raw;
+      const int rc = min(r, n_loc - 1);                      // clamped: no branch around the loads
       if (staged) {
 #pragma unroll
-        for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)r * LG + lane_in_row) * NW + w];
+        for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)rc * LG + lane_in_row) * NW + w];
       } else {
-        const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)(lo + r) * P.q_st + lane_in_row * 8);
+        const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)(lo + rc) * P.q_st + lane_in_row * 8);
 #pragma unroll
         for (int w = 0; w < NW; ++w) raw.w[w] = __ldg(src + w);
       }
       float x[8];
       raw_to_f32<T>(raw, x);
+      const float live = r < n_loc ? 1.f : 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { acc[i] += x[i]; nn = fmaf(x[i], x[i], nn); }
+      for (int i = 0; i < 8; ++i) { acc[i] = fmaf(x[i], live, acc[i]); nn = fmaf(x[i], x[i], nn); }
+#pragma unroll
+      for (int o = LG / 2; o > 0; o >>= 1) nn += __shfl_xor_sync(0xFFFFFFFFu, nn, o);
+      if (lane_in_row == 0 && r < n_loc) norms[r] = fmaxf(sqrtf(nn), kNormEps);
     }
-#pragma unroll
-    for (int o = LG / 2; o > 0; o >>= 1) nn += __shfl_xor_sync(0xFFFFFFFFu, nn, o);
-    if (lane_in_row == 0 && r < n_loc) norms[r] = fmaxf(sqrtf(nn), kNormEps);
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) red[row_slot * D + lane_in_row * 8 + i] = acc[i];
@@ -152,22 +176,21 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   const float mn = Mnorm;
   for (int r0 = 0; r0 < n_sort; r0 += RPI) {
     const int r = r0 + row_slot;
-    float dot = 0.f;
-    if (r < n_loc) {
-      Raw8<T> raw;
-      if (staged) {
+    const int rc = max(min(r, n_loc - 1), 0);             // clamped (an empty slice reads row 0 / the last row)
+    Raw8<T> raw;
+    if (staged) {
 #pragma unroll
-        for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)r * LG + lane_in_row) * NW + w];
-      } else {
-        const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)(lo + r) * P.q_st + lane_in_row * 8);
+      for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)rc * LG + lane_in_row) * NW + w];
+    } else {
+      const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)min(lo + rc, C - 1) * P.q_st + lane_in_row * 8);
 #pragma unroll
-        for (int w = 0; w < NW; ++w) raw.w[w] = __ldg(src + w);
-      }
-      float x[8];
-      raw_to_f32<T>(raw, x);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) dot = fmaf(x[i], m[i], dot);
+      for (int w = 0; w < NW; ++w) raw.w[w] = __ldg(src + w);
     }
+    float x[8];
+    raw_to_f32<T>(raw, x);
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) dot = fmaf(x[i], m[i], dot);
 #pragma unroll
     for (int o = LG / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
     if (lane_in_row == 0 && r < n_sort) {
@@ -181,44 +204,65 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   }
   __syncthreads();
 
-  // ---- bitonic sort of the slice, ascending
-  for (int k = 2; k <= n_sort; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < n_sort; i += kRankThreads) {
-        const int ixj = i ^ j;
-        if (ixj > i) {
-          const unsigned long long a = keys[i], b = keys[ixj];
-          const bool up = (i & k) == 0;
-          if ((a > b) == up) { keys[i] = b; keys[ixj] = a; }
-        }
+  // ---- sort of the slice, ascending.  Each warp sorts 32-key runs in registers (bitonic network over
+  // shuffles, no block barriers); then every key finds its place by counting the smaller keys of the other
+  // runs with branch-free binary searches (keys are unique) and is scattered to `sorted`.
+  const int lane = tid & 31, wid = tid >> 5;
+  const int n_runs = n_sort >> 5;
+  for (int run = wid; run < n_runs; run += kRankThreads / 32) {
+    unsigned long long v = keys[run * 32 + lane];
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
+        const bool up = (lane & k) == 0, lower = (lane & j) == 0;
+        const bool take_min = up == lower;
+        v = take_min ? (v < o ? v : o) : (v < o ? o : v);
       }
-      __syncthreads();
     }
+    keys[run * 32 + lane] = v;
+  }
+  for (int i = tid; i < n_sort; i += kRankThreads) sorted[i] = ~0ull;   // slots the padding keys do not reach
+  __syncthreads();
+  for (int i = tid; i < n_sort; i += kRankThreads) {
+    const unsigned long long key = keys[i];
+    const int my_run = i >> 5;
+    int rk = i & 31;
+#pragma unroll 1
+    for (int run = 0; run < n_runs; ++run) {
+      const unsigned long long* pr = keys + run * 32;
+      int pos = 0;
+#pragma unroll
+      for (int step = 16; step > 0; step >>= 1) pos += pr[pos + step - 1] < key ? step : 0;
+      pos += pr[pos] < key ? 1 : 0;
+      rk += run == my_run ? 0 : pos;
+    }
+    sorted[rk] = key;                                     // padding keys are equal: they may collide, all ~0
   }
   cluster.sync();                                         // every slice is sorted
 
   // ---- global rank of my N smallest: own rank + number of smaller codes in each peer's slice.  Only a
-  // peer's first m_peer = min(n_sort, N) codes matter (more smaller ones than that already push the rank past
-  // N); they are copied into local shared memory first, because a chain of dependent remote reads is slow.
+  // peer's first m_peer codes matter (m_peer = a power of two >= min(n_sort, N): more smaller ones than N
+  // already push the rank past N); they are copied into local shared memory first, because a chain of
+  // dependent remote reads is slow.
   for (int e = tid; e < (kRankCluster - 1) * m_peer; e += kRankThreads) {
     const int pr = e / m_peer, j = e % m_peer;
     const int r = pr + (pr >= rank ? 1 : 0);
-    peer_keys[e] = cluster.map_shared_rank(keys, r)[j];
+    peer_keys[e] = cluster.map_shared_rank(sorted, r)[j];
   }
   __syncthreads();
   const int n_cand = min(N, n_loc);
   for (int li = tid; li < n_cand; li += kRankThreads) {
-    const unsigned long long key = keys[li];
+    const unsigned long long key = sorted[li];
     int rk = li;
 #pragma unroll 1
     for (int pr = 0; pr < kRankCluster - 1; ++pr) {
       const unsigned long long* pk = peer_keys + (size_t)pr * m_peer;
-      int a = 0, b = m_peer;                              // first index with pk[idx] >= key
-      while (a < b) {
-        const int mid = (a + b) >> 1;
-        if (pk[mid] < key) a = mid + 1; else b = mid;
-      }
-      rk += a;
+      int pos = 0;                                        // number of pk[] entries below key, branch-free
+      for (int step = m_peer >> 1; step > 0; step >>= 1) pos += pk[pos + step - 1] < key ? step : 0;
+      pos += pk[pos] < key ? 1 : 0;
+      rk += pos;
     }
     if (rk < N) out[rk] = (int32_t)(key & 0xFFFFFFFFull);
   }
@@ -284,11 +328,12 @@ template <typename T, int D>
 static cudaError_t launch_rank_t(const DevParams& P, const void* q, int32_t* q_idx, cudaStream_t st) {
   constexpr int LG = D / 8, RPI = kRankThreads / LG;
   int rpc = (P.chunk + kRankCluster - 1) / kRankCluster;
-  int n_sort = 2;
+  int n_sort = 32;
   while (n_sort < rpc) n_sort <<= 1;
   const size_t row_bytes = (size_t)rpc * D * sizeof(T);
-  const int m_peer = n_sort < P.n_sel ? n_sort : P.n_sel;
-  const size_t fixed = (size_t)n_sort * 8 + (size_t)RPI * D * 4 + (size_t)((rpc + 3) & ~3) * 4 + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1) * 8;
+  int m_peer = 1;
+  while (m_peer < P.n_sel && m_peer < n_sort) m_peer <<= 1;
+  const size_t fixed = (size_t)n_sort * 16 + (size_t)RPI * D * 4 + (size_t)((rpc + 3) & ~3) * 4 + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1) * 8;
   const int staged = fixed + row_bytes <= kRankStageLimit + 48 * 1024 && row_bytes <= kRankStageLimit ? 1 : 0;
   const size_t smem = fixed + (staged ? row_bytes : 0);
   cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
