@@ -30,6 +30,9 @@ import torch  # noqa: E402
 
 METRIC = "us_per_prefill_chunk"
 UNIT = "us"
+# DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu capture of that workload
+# (profiles/kernels_full_<workload>.md); None where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {("llama8b_32k", "sparse_attn"): 42.9e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -406,7 +409,8 @@ def main():
     staged_sum = sum(kernels[n]["us"] for n in stages)
     dom = "sparse_attn"
     roofline = {"kernel": dom, "bound": "tensor", "achieved": kernels[dom]["tflops"], "peak": pk["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": kernels[dom]["frac"], "traffic": None,
+                "unit": "TFLOP/s", "frac": kernels[dom]["frac"],
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom)),
                 "peak_source": f"{pk['source']} burst bf16 (kernel timed alone)"}
 
     # ---- end to end through the host-buffer entry point (contiguous caches only)
