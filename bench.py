@@ -230,6 +230,80 @@ def host_threads():
         return os.cpu_count() or 1
 
 
+# ----------------------------------------------------------------------------- whole-prompt sweep
+def sweep(args, w, q, k, v, out, ctx, dev, rank):
+    """Algorithm 2 over a whole prompt of T + C tokens: chunk i sees T_i = i*C cached rows (the synthetic cache rows
+    stand in for the keys earlier chunks would have appended).  Budget = 12 % of the cached length per chunk."""
+    from paper_2602_08722_b200 import api
+    T, C = w["T"], w["C"]
+    lens = list(range(0, T + 1, C))
+    frac = 0.12
+    ps = [api.make_params(q, k, out, ctx, n_retain=w["n_retain"], kv_budget=0, budget_frac=frac, max_ctx_len=t)
+          for t in lens]
+    for p_i in ps:
+        p_i.kv_rows = k.shape[2]
+    ws = api.alloc_workspace(ps[-1])
+    len_dev = [torch.tensor([t], dtype=torch.int32, device=dev) for t in lens]
+
+    def chunk(i, dense):
+        ctx.copy_(len_dev[i])                                   # device-to-device on the stream: graph-safe
+        if dense:
+            api.quoka_dense_chunk_attn(ps[i], q, k, v, out, None, ws)
+        else:
+            api.quoka_prefill_chunk(ps[i], q, k, v, out, None, None, ws)
+
+    def run(dense):
+        for i in range(len(lens)):
+            chunk(i, dense)
+
+    def timed(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.mean(ts)
+
+    n0 = api.quoka_launch_count()
+    eager_us = timed(lambda: run(False), 5)
+    launches = (api.quoka_launch_count() - n0) // 6
+    per_chunk = []
+    for i in range(len(lens)):
+        per_chunk.append(round(timed(lambda: chunk(i, False), 3), 1))
+    dense_us = timed(lambda: run(True), 2)
+    graph_us = None
+    try:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            run(False)                                          # warm-up on the capture stream
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                run(False)
+        torch.cuda.synchronize()
+        graph_us = timed(g.replay, 5)
+    except Exception as e:                                      # capture not possible: report it, keep the eager number
+        graph_us = None
+        graph_err = repr(e)[:200]
+    status = api.quoka_last_device_status(ws)
+    if rank == 0:
+        line = {"metric": "us_per_prompt_prefill_attention", "value": round(eager_us, 1), "unit": "us",
+                "config": {"workload": args.workload, "chunks": len(lens), "chunk_len": C, "final_ctx_len": T,
+                           "budget_frac": frac, "n_retain": w["n_retain"]},
+                "sweep": {"quoka_eager_us": round(eager_us, 1), "quoka_graph_us": None if graph_us is None else round(graph_us, 1),
+                          "dense_us": round(dense_us, 1), "speedup_vs_dense": round(dense_us / eager_us, 3),
+                          "per_chunk_us": per_chunk, "gpu_launches_per_sweep": launches},
+                "device_status": status, "note": "sweep mode (Algorithm 2 over the whole prompt); not the default bench line"}
+        if graph_us is None:
+            line["sweep"]["graph_error"] = graph_err
+        print(json.dumps(line))
+    return 0
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -243,6 +317,9 @@ def main():
     ap.add_argument("--fused-only", action="store_true",
                     help="only the timed fused steps (for profiler captures): no per-kernel, e2e or CPU legs")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--sweep", action="store_true",
+                    help="chunked prefill of the whole prompt (Algorithm 2): chunks at cached lengths 0, C, 2C, .. T, "
+                         "eager launches and one CUDA graph, against the dense chunk kernel; prints its own JSON line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -326,6 +403,9 @@ def main():
             import torch.distributed as dist
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.sweep:
+        return sweep(args, w, q, k, v, out, ctx, dev, rank)
 
     def step():
         api.quoka_prefill_chunk(p, q, k, v, out, None, None, ws)

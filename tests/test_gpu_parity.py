@@ -223,3 +223,45 @@ def test_sweep_points_32k(pt):
                  budget_frac=c["budget_frac"])
     gp.run_staged()
     check_chain(gp, attn_rows=64)
+
+
+# ---------------------------------------------------------------- Algorithm 2 as a loop over chunks, eager and as one CUDA graph
+def test_chunk_loop_replayed_from_a_cuda_graph_matches_eager_calls():
+    # the same buffers serve every chunk; only the cached length (a device tensor) and the host bound change
+    T_max, C = 1536, 256
+    inp = synth.make_chunk_inputs(12, 1, 8, 2, 128, T_max, C, "bf16")
+    gp = GpuProblem(inp, 32, kv_budget=0, budget_frac=0.25)
+    lens = [0, 512, 1024, 1536]
+    ps = [api.make_params(gp.q, gp.k, gp.out, gp.ctx_len, n_retain=32, budget_frac=0.25, max_ctx_len=t) for t in lens]
+    len_dev = [torch.tensor([t], dtype=torch.int32, device="cuda") for t in lens]
+    outs = [torch.zeros_like(gp.out) for _ in lens]
+
+    def run():
+        for i in range(len(lens)):
+            gp.ctx_len.copy_(len_dev[i])
+            api.quoka_prefill_chunk(ps[i], gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+            outs[i].copy_(gp.out)
+
+    run()
+    torch.cuda.synchronize()
+    want = [o.clone() for o in outs]
+    # chunk 0 (empty cache) is plain causal self-attention over rows [0, C): checked against the oracle
+    q = f64(gp.inp.q[0])
+    dense0, _ = O.dense_chunk_attention(q, f64(gp.inp.k[0, :, :C]), f64(gp.inp.v[0, :, :C]), 0)
+    check_attention(f64(want[0][0]), dense0, "bf16")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run()
+        side.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            run()
+    torch.cuda.synchronize()
+    for o in outs:
+        o.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(outs, want):
+        assert torch.equal(a, b)
+    assert api.quoka_last_device_status(gp.ws) == 0
