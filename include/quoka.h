@@ -71,6 +71,17 @@ typedef enum {
   QUOKA_IMPL_TENSOR = 2  /* tcgen05 kernels; QUOKA_ERR_UNSUPPORTED if dtype is f32 */
 } quoka_impl;
 
+/* How a cached key is scored against the retained queries (the paper's ablations, Appendix "Ablations").
+ * The defaults are the method as published: cosine similarity, maximum over the retained queries. */
+typedef enum {
+  QUOKA_SCORE_COSINE = 0,  /* Alg. 1: queries and keys divided by their norms before the product          */
+  QUOKA_SCORE_DOT = 1      /* ablation: raw dot products, neither queries nor keys are normalised         */
+} quoka_score_mode;
+typedef enum {
+  QUOKA_AGG_MAX = 0,       /* Alg. 1: S^ = max over the retained queries                                  */
+  QUOKA_AGG_MEAN = 1       /* ablation: S^ = mean over the retained queries                               */
+} quoka_query_agg;
+
 typedef struct {
   int32_t batch, n_q_heads, n_kv_heads, head_dim;
   int32_t chunk_len;     /* C = B_CP                                                          */
@@ -92,6 +103,8 @@ typedef struct {
   int64_t kv_stride_b, kv_stride_h, kv_stride_t;   /* kv_stride_b is the page stride when paged */
   int64_t kv_rows;             /* rows allocated per (sequence, head) when contiguous (>= T_s+C);
                                   number of pages in the pool when paged                        */
+  int32_t score_mode;          /* quoka_score_mode; affects qbar (normalised or raw) and the scores */
+  int32_t query_agg;           /* quoka_query_agg                                                 */
 } quoka_params;
 
 /* Row pitch of k_idx: the largest B_s any sequence can have, from max_ctx_len. */

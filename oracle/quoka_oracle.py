@@ -108,36 +108,50 @@ def select_queries(q, n_retain):
 # --------------------------------------------------------------------------
 # Algorithm 1, "Efficient Cosine Similarity via Pre-aggregation"
 # --------------------------------------------------------------------------
-def aggregate_queries(q, q_idx, n_kv, storage="f32"):
+def aggregate_queries(q, q_idx, n_kv, storage="f32", score_mode="cosine"):
     """Q <- gather(Q, idx); Q <- Q / norm(Q); Q-bar <- mean over the G heads of
     each KV group of the rank-aligned retained queries.  (n_KV, N, d).
     With storage == "bf16" Q-bar is rounded once to bfloat16, because it is
-    stored in the cache dtype before the scoring product."""
+    stored in the cache dtype before the scoring product.
+    score_mode == "dot" is the ablation of the Appendix "Ablations" (dot
+    products instead of cosine similarity): the division by the norm is left
+    out, everything else is unchanged."""
     q = np.asarray(q, dtype=np.float64)
     n_q, C, d = q.shape
     G = n_q // n_kv
     assert G * n_kv == n_q
     N = q_idx.shape[1]
     gathered = np.take_along_axis(q, q_idx.astype(np.int64)[:, :, None], axis=1)  # (n_Q, N, d)
-    norms = np.maximum(np.sqrt((gathered * gathered).sum(axis=2, keepdims=True)), EPS)
-    q_hat = gathered / norms
+    assert score_mode in ("cosine", "dot")
+    if score_mode == "cosine":
+        norms = np.maximum(np.sqrt((gathered * gathered).sum(axis=2, keepdims=True)), EPS)
+        q_hat = gathered / norms
+    else:
+        q_hat = gathered
     qbar = q_hat.reshape(n_kv, G, N, d).mean(axis=1)
     if storage == "bf16":
         qbar = round_to_bf16(qbar)
     return qbar
 
 
-def score_keys(qbar, k, T):
+def score_keys(qbar, k, T, score_mode="cosine", query_agg="max"):
     """K <- K / norm(K); S <- Q-bar K^T; S-hat <- max(S, dim=queries).
-    qbar: (n_KV, N, d); k: (n_KV, >=T, d).  Returns (n_KV, T)."""
+    qbar: (n_KV, N, d); k: (n_KV, >=T, d).  Returns (n_KV, T).
+    The two ablations of the Appendix "Ablations": score_mode == "dot" leaves
+    the keys un-normalised; query_agg == "mean" takes the mean over the query
+    axis instead of the maximum."""
+    assert score_mode in ("cosine", "dot") and query_agg in ("max", "mean")
     qbar = np.asarray(qbar, dtype=np.float64)
     kc = np.asarray(k, dtype=np.float64)[:, :T, :]
-    kn = np.maximum(np.sqrt((kc * kc).sum(axis=2, keepdims=True)), EPS)
-    k_hat = kc / kn
+    if score_mode == "cosine":
+        kn = np.maximum(np.sqrt((kc * kc).sum(axis=2, keepdims=True)), EPS)
+        k_hat = kc / kn
+    else:
+        k_hat = kc
     S = qbar @ np.swapaxes(k_hat, 1, 2)                       # (n_KV, N, T)
     if S.shape[1] == 0:
         return np.full((kc.shape[0], T), -np.inf)
-    return S.max(axis=1)
+    return S.max(axis=1) if query_agg == "max" else S.mean(axis=1)
 
 
 def select_keys(scores, B):
@@ -229,15 +243,15 @@ def sparse_attention_rows(q, k, v, T, k_idx, heads, rows, scale=None):
 # the whole per-chunk path
 # --------------------------------------------------------------------------
 def quoka_prefill_chunk(q, k, v, T, n_retain, kv_budget=0, budget_frac=0.0,
-                        storage="f32", scale=None):
+                        storage="f32", scale=None, score_mode="cosine", query_agg="max"):
     """Algorithm 2, loop body, for one sequence: select queries, score and select
     cached keys, attend.  Returns a dict with every intermediate."""
     n_kv = np.asarray(k).shape[0]
     T = int(T)
     B = key_budget(T, kv_budget, budget_frac)
     q_idx, cos = select_queries(q, n_retain)
-    qbar = aggregate_queries(q, q_idx, n_kv, storage)
-    scores = score_keys(qbar, k, T)
+    qbar = aggregate_queries(q, q_idx, n_kv, storage, score_mode)
+    scores = score_keys(qbar, k, T, score_mode, query_agg)
     k_idx = select_keys(scores, B)
     out, lse = sparse_attention(q, k, v, T, k_idx, scale)
     return dict(q_idx=q_idx, cos=cos, qbar=qbar, scores=scores, k_idx=k_idx,

@@ -19,6 +19,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_
 STATIC_SCRATCH_BYTES = 8 << 20
 BF16, F32 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
+SCORE_COSINE, SCORE_DOT = 0, 1
+AGG_MAX, AGG_MEAN = 0, 1
 
 EXPORTS = [
     "quoka_kv_budget_cap", "quoka_workspace_size", "quoka_select_queries", "quoka_score_keys",
@@ -44,6 +46,7 @@ class QuokaParams(C.Structure):
         ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32), ("block_table", C.c_void_p),
         ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_t", C.c_int64),
         ("kv_rows", C.c_int64),
+        ("score_mode", C.c_int32), ("query_agg", C.c_int32),
     ]
 
 
@@ -106,7 +109,8 @@ def _check(status: int, where: str):
 
 
 def make_params(q, k_cache, out, ctx_len, *, n_retain, kv_budget=0, budget_frac=0.0, max_ctx_len,
-                block_table=None, impl=IMPL_AUTO, softmax_scale=0.0) -> QuokaParams:
+                block_table=None, impl=IMPL_AUTO, softmax_scale=0.0, score_mode=SCORE_COSINE,
+                query_agg=AGG_MAX) -> QuokaParams:
     """Fill quoka_params from tensors: q/out (b, n_Q, C, d); k_cache (b, n_KV, rows, d)
     contiguous or (pages, n_KV, 64, d) with a block table (b, max_pages)."""
     b, n_q, c, d = q.shape
@@ -116,6 +120,7 @@ def make_params(q, k_cache, out, ctx_len, *, n_retain, kv_budget=0, budget_frac=
     p.kv_budget, p.budget_frac = int(kv_budget), float(budget_frac)
     p.dtype = BF16 if q.dtype == torch.bfloat16 else F32
     p.impl, p.softmax_scale, p.max_ctx_len = int(impl), float(softmax_scale), int(max_ctx_len)
+    p.score_mode, p.query_agg = int(score_mode), int(query_agg)
     p.ctx_len = ctx_len.data_ptr()
     p.q_stride_b, p.q_stride_h, p.q_stride_t = q.stride(0), q.stride(1), q.stride(2)
     p.o_stride_b, p.o_stride_h, p.o_stride_t = out.stride(0), out.stride(1), out.stride(2)

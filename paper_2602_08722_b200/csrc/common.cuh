@@ -30,6 +30,8 @@ struct DevParams {
   const int32_t* block_table;
   int64_t kv_sb, kv_sh, kv_st;
   int32_t* status;  // device status word
+  int score_dot;    // 1: raw dot products (no normalisation of queries or keys)
+  int agg_mean;     // 1: mean over the retained queries instead of the maximum
 };
 
 // B_s of one sequence: min(B_SA, T) or floor(frac*T + 0.5) in double.

@@ -61,6 +61,8 @@ static quoka_status validate(const quoka_params* p) {
   if (p->kv_budget <= 0 && !(p->budget_frac >= 0.f && p->budget_frac <= 1.f)) return QUOKA_ERR_INVALID_ARG;
   if (p->dtype != QUOKA_BF16 && p->dtype != QUOKA_F32) return QUOKA_ERR_INVALID_ARG;
   if (p->impl < QUOKA_IMPL_AUTO || p->impl > QUOKA_IMPL_TENSOR) return QUOKA_ERR_INVALID_ARG;
+  if (p->score_mode < QUOKA_SCORE_COSINE || p->score_mode > QUOKA_SCORE_DOT) return QUOKA_ERR_INVALID_ARG;
+  if (p->query_agg < QUOKA_AGG_MAX || p->query_agg > QUOKA_AGG_MEAN) return QUOKA_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return QUOKA_ERR_UNSUPPORTED;
   if (p->page_size != 0 && p->page_size != kPage) return QUOKA_ERR_UNSUPPORTED;
   if (p->page_size == kPage && (!p->block_table || p->max_pages_per_seq <= 0)) return QUOKA_ERR_INVALID_ARG;
@@ -100,6 +102,8 @@ static DevParams make_dev(const quoka_params* p, void* ws) {
   P.page_size = p->page_size; P.max_pages = p->max_pages_per_seq; P.block_table = p->block_table;
   P.kv_sb = p->kv_stride_b; P.kv_sh = p->kv_stride_h; P.kv_st = p->kv_stride_t;
   P.status = static_cast<int32_t*>(ws);
+  P.score_dot = p->score_mode == QUOKA_SCORE_DOT ? 1 : 0;
+  P.agg_mean = p->query_agg == QUOKA_AGG_MEAN ? 1 : 0;
   return P;
 }
 

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kScoreTile) score_keys_simt_kernel(DevParams P
   for (int x = 0; x < D; ++x) nn += krow[x] * krow[x];
 
   const E* qb = qbar + ((int64_t)s * P.n_kv + kv) * (int64_t)N * D;
-  float best = -INFINITY;
+  float best = -INFINITY, total = 0.f;
   for (int j0 = 0; j0 < N; j0 += kQChunk) {
     const int nq = min(kQChunk, N - j0);
     __syncthreads();
@@ -63,10 +63,11 @@ __global__ void __launch_bounds__(kScoreTile) score_keys_simt_kernel(DevParams P
     }
 #pragma unroll
     for (int j = 0; j < kQChunk; ++j)
-      if (j < nq) best = fmaxf(best, acc[j]);
+      if (j < nq) { best = fmaxf(best, acc[j]); total += acc[j]; }
   }
   if (t0 + tid < T)
-    scores[((int64_t)s * P.n_kv + kv) * P.max_ctx + t0 + tid] = best / fmaxf(sqrtf(nn), kNormEps);
+    scores[((int64_t)s * P.n_kv + kv) * P.max_ctx + t0 + tid] =
+        (P.agg_mean ? total / (float)N : best) / (P.score_dot ? 1.f : fmaxf(sqrtf(nn), kNormEps));
 }
 
 cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,

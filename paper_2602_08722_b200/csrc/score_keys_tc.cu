@@ -252,6 +252,8 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
       if (!mbar_wait(&acc_full[slot], acc_phase, wc)) break;
       tc_fence_after();
       float bacc[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      float sacc[4] = {0.f, 0.f, 0.f, 0.f};               // mean-over-queries variant: columns >= N are exact zeros
+      const bool agg_mean = P.agg_mean != 0;
       for (int p = 0; p < A.n_parts; ++p) {
         const int n_mma = (p == A.n_parts - 1) ? (A.n_pad - p * 256) : 256;
         const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((A.n_parts == 1 ? slot : p) * 256);
@@ -261,6 +263,10 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
           tmem_ld32(t_addr + c0, r0);
           tmem_ld32(t_addr + c0 + 32, r1);
           tmem_wait_ld();
+          if (agg_mean) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sacc[j & 3] += __uint_as_float(r0[j]) + __uint_as_float(r1[j]);
+          }
           const int lim = A.n - (p * 256 + c0);
           if (lim >= 64) {
 #pragma unroll
@@ -277,6 +283,10 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
           uint32_t r[32];
           tmem_ld32(t_addr + c0, r);
           tmem_wait_ld();
+          if (agg_mean) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sacc[j & 3] += __uint_as_float(r[j]);
+          }
           const int lim = A.n - (p * 256 + c0);
 #pragma unroll
           for (int j = 0; j < 32; ++j)
@@ -286,19 +296,24 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
           uint32_t r[16];
           tmem_ld16(t_addr + c0, r);
           tmem_wait_ld();
+          if (agg_mean) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) sacc[j & 3] += __uint_as_float(r[j]);
+          }
           const int lim = A.n - (p * 256 + c0);
 #pragma unroll
           for (int j = 0; j < 16; ++j)
             if (j < lim) bacc[j & 3] = fmaxf(bacc[j & 3], __uint_as_float(r[j]));
         }
       }
-      const float best = fmaxf(fmaxf(bacc[0], bacc[1]), fmaxf(bacc[2], bacc[3]));
+      const float best = agg_mean ? ((sacc[0] + sacc[1]) + (sacc[2] + sacc[3])) / (float)A.n
+                                  : fmaxf(fmaxf(bacc[0], bacc[1]), fmaxf(bacc[2], bacc[3]));
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[slot]);
       const int t = w.tile * kTileKeys + row;
       if (t < __ldg(P.ctx_len + w.s))
-        scores[((long long)w.s * P.n_kv + w.kv) * P.max_ctx + t] = best / fmaxf(sqrtf(nn), kNormEps);
+        scores[((long long)w.s * P.n_kv + w.kv) * P.max_ctx + t] = P.score_dot ? best : best / fmaxf(sqrtf(nn), kNormEps);
       if (++stage == A.stages) { stage = 0; phase ^= 1; }
     }
   }

@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, con
 #pragma unroll
         for (int i = 0; i < NE; ++i) nn += x[u][i] * x[u][i];
         nn = warp_sum(nn);
-        const float norm = fmaxf(sqrtf(nn), kNormEps);
+        const float norm = P.score_dot ? 1.f : fmaxf(sqrtf(nn), kNormEps);
         if (g4 + u < g_end) {
 #pragma unroll
           for (int i = 0; i < NE; ++i) acc[i] += x[u][i] / norm;

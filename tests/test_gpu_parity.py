@@ -13,11 +13,13 @@ IMPLS = [pytest.param(api.IMPL_SIMT, id="simt"), pytest.param(api.IMPL_AUTO, id=
 
 
 def problem(seed, *, batch=1, n_q=4, n_kv=2, d=128, T=1000, C=300, dtype="bf16", n_retain=24, kv_budget=177,
-            budget_frac=0.0, impl=api.IMPL_AUTO, paged=False, capacity=None, max_ctx_len=None):
+            budget_frac=0.0, impl=api.IMPL_AUTO, paged=False, capacity=None, max_ctx_len=None, score_mode="cosine",
+            query_agg="max"):
     inp = synth.make_chunk_inputs(seed, batch, n_q, n_kv, d, T, C, dtype, capacity=capacity)
     if paged:
         inp = synth.to_paged(inp, seed)
-    return GpuProblem(inp, n_retain, kv_budget, budget_frac, impl=impl, paged=paged, max_ctx_len=max_ctx_len)
+    return GpuProblem(inp, n_retain, kv_budget, budget_frac, impl=impl, paged=paged, max_ctx_len=max_ctx_len,
+                      score_mode=score_mode, query_agg=query_agg)
 
 
 # ---------------------------------------------------------------- small cases, every stage, all rows
@@ -78,6 +80,27 @@ def test_batched_variable_lengths(paged, impl):
 
 def test_max_ctx_len_may_exceed_every_sequence():
     gp = problem(6, T=600, C=128, capacity=2048, max_ctx_len=1500, kv_budget=0, budget_frac=0.5)
+    gp.run_staged()
+    check_chain(gp)
+
+
+# ---------------------------------------------------------------- ablation variants of the scoring step
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("score_mode,query_agg", [("dot", "max"), ("cosine", "mean"), ("dot", "mean")])
+def test_scoring_ablation_variants(score_mode, query_agg, dtype, impl):
+    gp = problem(13, n_q=8, n_kv=2, T=1500, C=290, dtype=dtype, n_retain=40, kv_budget=300, impl=impl,
+                 score_mode=score_mode, query_agg=query_agg)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(staged, gp.out)
+
+
+def test_scoring_ablation_with_more_than_256_retained_queries():
+    gp = problem(14, n_q=4, n_kv=2, T=900, C=700, n_retain=300, kv_budget=200, score_mode="dot", query_agg="mean")
     gp.run_staged()
     check_chain(gp)
 

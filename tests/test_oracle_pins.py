@@ -92,6 +92,46 @@ def test_algorithm1_hand_example():
                                   g["k_idx_head0_alone_B2"])
 
 
+def test_ablation_variants_hand_example_and_invariants():
+    """Dot-product scoring and mean-over-queries aggregation (Appendix "Ablations")."""
+    g = _load_golden()
+    q = np.stack([g["q_head0"].reshape(4, 2), g["q_head1"].reshape(4, 2)])
+    k = g["k"].reshape(1, 4, 2)
+    q_idx = np.stack([g["q_idx_head0"], g["q_idx_head1"]]).astype(np.int32)
+    # head 0 alone, raw dot products: table values
+    qb = O.aggregate_queries(q[:1], q_idx[:1], n_kv=1, score_mode="dot")
+    np.testing.assert_allclose(qb[0], q[0][[3, 0]], atol=0)              # raw retained rows, no normalisation
+    np.testing.assert_allclose(O.score_keys(qb, k, 4, "dot", "max")[0], g["dot_max_head0_alone"], atol=1e-9)
+    np.testing.assert_allclose(O.score_keys(qb, k, 4, "dot", "mean")[0], g["dot_mean_head0_alone"], atol=1e-9)
+    # both heads, cosine scoring, mean over the two ranks
+    qbar = O.aggregate_queries(q, q_idx, n_kv=1)
+    np.testing.assert_allclose(O.score_keys(qbar, k, 4, "cosine", "mean")[0], g["cos_mean"], atol=1e-9)
+    # invariants on random data: dot scores are linear in the key, cosine scores ignore its length;
+    # mean <= max; one retained query makes mean == max; dot/max with G = 1 is a plain matrix product
+    qr, kr, _ = rand_problem(5, n_q=4, n_kv=2, C=9, d=8, T=13)
+    idx, _ = O.select_queries(qr, 3)
+    for mode in ("cosine", "dot"):
+        qb = O.aggregate_queries(qr, idx, 2, score_mode=mode)
+        mx = O.score_keys(qb, kr, 13, mode, "max")
+        mn = O.score_keys(qb, kr, 13, mode, "mean")
+        assert (mn <= mx + 1e-12).all()
+        k2 = kr.copy()
+        k2[:, 5] *= 3.0
+        mx2 = O.score_keys(qb, k2, 13, mode, "max")
+        want = mx.copy()
+        if mode == "dot":
+            want[:, 5] *= 3.0
+        np.testing.assert_allclose(mx2, want, atol=1e-12)
+        one = O.score_keys(qb[:, :1], kr, 13, mode, "mean")
+        np.testing.assert_allclose(one, O.score_keys(qb[:, :1], kr, 13, mode, "max"), atol=1e-12)
+    idx1 = np.tile(np.arange(9), (4, 1)).astype(np.int32)                 # all queries, G = 1
+    qb = O.aggregate_queries(qr, idx1, 4, score_mode="dot")
+    dots = np.stack([qr[h] @ kr[h // 2, :13].T for h in range(4)])        # (4, C, T), written out per head
+    kr4 = np.stack([kr[h // 2] for h in range(4)])
+    got = O.score_keys(qb, kr4, 13, "dot", "max")
+    np.testing.assert_allclose(got, dots.max(axis=1), atol=1e-12)
+
+
 # ------------------------------------------------------------------ query sub-selection
 def test_query_cosines_match_library_cosine_distance():
     q, _, _ = rand_problem(1, n_q=3, C=17, d=8)
@@ -407,6 +447,9 @@ MUTANTS = {
     "wrong kv head for attention": ("        kv = h // G\n        idx = np.asarray(k_idx[kv], dtype=np.int64)\n        out[h]", "        kv = h % n_kv\n        idx = np.asarray(k_idx[kv], dtype=np.int64)\n        out[h]"),
     "renormalised qbar": ("    if storage == \"bf16\":\n        qbar = round_to_bf16(qbar)\n    return qbar", "    qbar = qbar / np.sqrt((qbar*qbar).sum(axis=2, keepdims=True))\n    return qbar"),
     "truncating bf16": ("rounded = (bits + np.uint64(0x7FFF) + lsb)", "rounded = (bits)"),
+    "dot mode normalises keys": ("    else:\n        k_hat = kc", "    else:\n        k_hat = kc / np.sqrt((kc * kc).sum(axis=2, keepdims=True))"),
+    "dot mode normalises queries": ("    else:\n        q_hat = gathered", "    else:\n        q_hat = gathered / np.sqrt((gathered * gathered).sum(axis=2, keepdims=True))"),
+    "mean mode sums": ("else S.mean(axis=1)", "else S.sum(axis=1)"),
 }
 
 PIN_TESTS = [
@@ -419,7 +462,7 @@ PIN_TESTS = [
     test_empty_cache_is_causal_self_attention_and_row0_is_v0,
     test_identical_keys_give_uniform_average_of_visible_values,
     test_full_budget_and_all_queries_equals_dense, test_query_cosines_match_library_cosine_distance,
-    test_selection_invariant_to_positive_rescaling,
+    test_selection_invariant_to_positive_rescaling, test_ablation_variants_hand_example_and_invariants,
 ]
 
 
