@@ -113,6 +113,9 @@ WORKLOADS = {
     "tiny_f32": dict(batch=1, n_q=8, n_kv=2, d=128, T=4096, C=256, n_retain=32, kv_budget=512, dtype="f32"),
     "llama8b_32k": dict(batch=1, n_q=32, n_kv=8, d=128, T=32768, C=2048, n_retain=128, kv_budget=3932, dtype="bf16"),
     "long_128k": dict(batch=1, n_q=32, n_kv=8, d=128, T=131072, C=4096, n_retain=256, kv_budget=15729, dtype="bf16"),
+    # generation phase (one query per sequence, no query sub-selection), budget 256 keys
+    "decode_32k": dict(batch=1, n_q=32, n_kv=8, d=128, T=32768, C=1, n_retain=16, kv_budget=256, dtype="bf16"),
+    "decode_32k_b16": dict(batch=16, n_q=32, n_kv=8, d=128, T=32768, C=1, n_retain=16, kv_budget=256, dtype="bf16"),
     "serving_mix": dict(batch=8, n_q=32, n_kv=8, d=128, T=None, C=1024, n_retain=64, kv_budget=0,
                         budget_frac=0.12, paged=True, dtype="bf16"),
 }

@@ -84,6 +84,30 @@ def test_max_ctx_len_may_exceed_every_sequence():
     check_chain(gp)
 
 
+# ---------------------------------------------------------------- generation phase: one query, no query sub-selection
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("paged", [False, True])
+def test_decode_step_single_query_per_sequence(paged, impl):
+    # a chunk of one query: Alg. 1 skips the sub-selection (C <= N_Q), Qbar is the group mean of the
+    # normalised query, the budget selects among the cached keys, the query attends them and itself
+    gp = problem(15, batch=3, n_q=8, n_kv=2, T=[2100, 333, 1290], C=1, n_retain=16, kv_budget=128, impl=impl,
+                 paged=paged)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(staged, gp.out)
+
+
+def test_decode_step_full_size_32k():
+    w = synth.WORKLOADS["decode_32k"]
+    gp = problem(0, n_q=w["n_q"], n_kv=w["n_kv"], d=w["d"], T=w["T"], C=w["C"], n_retain=w["n_retain"],
+                 kv_budget=w["kv_budget"])
+    gp.run_staged()
+    check_chain(gp)
+
+
 # ---------------------------------------------------------------- ablation variants of the scoring step
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
