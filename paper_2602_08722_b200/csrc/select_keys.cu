@@ -176,6 +176,8 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
     const int nb = pass == 2 ? 256 : kRegBins;
     uint32_t* hist = hist_all + pass * kRegBins;
+    // (compacting the threshold bin's rows into a list for the later passes was tried: building the list
+    // costs as much as the two passes it shortens)
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       const bool live = (base + 32 * i < T) && ((code[i] & mask) == prefix);
@@ -262,6 +264,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   }
   if (CL > 1) cluster.sync(); else __syncthreads();
   uint32_t run_gt = warp_off[wid], run_eq = warp_val[wid];
+  uint32_t total_eq = cta_cnt[1];
   if (CL > 1) {
     uint32_t pg[CL], pe[CL];
 #pragma unroll
@@ -270,21 +273,37 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
       pg[r] = pc[0];
       pe[r] = pc[1];
     }
+    total_eq = 0;
 #pragma unroll
-    for (int r = 0; r < CL; ++r)
+    for (int r = 0; r < CL; ++r) {
+      total_eq += pe[r];
       if (r < rank) { run_gt += pg[r]; run_eq += pe[r]; }
+    }
   }
+  if (need == total_eq) {
+    // every row equal to the threshold is taken (no tie is cut): one predicate, one ballot per item
+    uint32_t run = run_gt + run_eq;
 #pragma unroll
-  for (int i = 0; i < ITEMS; ++i) {
-    const int pos = base + 32 * i;
-    const bool in = pos < T;
-    const bool gt = in && code[i] > thr, eq = in && code[i] == thr;
-    const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt), b_eq = __ballot_sync(0xFFFFFFFFu, eq);
-    const uint32_t gt_before = run_gt + (uint32_t)__popc(b_gt & lt);
-    const uint32_t eq_before = run_eq + (uint32_t)__popc(b_eq & lt);
-    if (gt || (eq && eq_before < need)) out[gt_before + min(eq_before, need)] = pos;
-    run_gt += (uint32_t)__popc(b_gt);
-    run_eq += (uint32_t)__popc(b_eq);
+    for (int i = 0; i < ITEMS; ++i) {
+      const int pos = base + 32 * i;
+      const bool sel = pos < T && code[i] >= thr;
+      const uint32_t b = __ballot_sync(0xFFFFFFFFu, sel);
+      if (sel) out[run + (uint32_t)__popc(b & lt)] = pos;
+      run += (uint32_t)__popc(b);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+      const int pos = base + 32 * i;
+      const bool in = pos < T;
+      const bool gt = in && code[i] > thr, eq = in && code[i] == thr;
+      const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt), b_eq = __ballot_sync(0xFFFFFFFFu, eq);
+      const uint32_t gt_before = run_gt + (uint32_t)__popc(b_gt & lt);
+      const uint32_t eq_before = run_eq + (uint32_t)__popc(b_eq & lt);
+      if (gt || (eq && eq_before < need)) out[gt_before + min(eq_before, need)] = pos;
+      run_gt += (uint32_t)__popc(b_gt);
+      run_eq += (uint32_t)__popc(b_eq);
+    }
   }
   if (CL > 1) cluster.sync();                   // histograms and counts stay mapped until every peer has read them
 }
