@@ -76,6 +76,32 @@ def sum_work(w, ctx_lens):
     return tot
 
 
+# ----------------------------------------------------------------------------- ranks
+# The path shards with no exchange (every step is independent per sequence and KV head), so with N ranks each rank
+# runs its own independent chunk: the only cross-rank traffic is the barrier and the max over ranks of the time.
+def rank_workload(w, seed, rank):
+    """(seed of this rank's inputs, cached lengths of its sequences): ranks draw different problems."""
+    from paper_2602_08722_b200 import synth
+    if w["T"] is None:
+        return seed + rank, synth.serving_mix_ctx_lens(seed + rank, w["batch"])
+    return seed + rank, [w["T"]] * w["batch"]
+
+
+def max_over_ranks(x, world, device=None):
+    """Max over the ranks of a host float (the slowest rank decides); the value itself with one rank."""
+    if world <= 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_us_per_chunk(total_us, steps, world):
+    """Whole-job metric: every rank processed `steps` chunks in `total_us` (max over ranks)."""
+    return total_us / (steps * world)
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """SM clock and throttle-reason samples taken while the timed region runs: NVML every 5 ms in a thread
@@ -328,10 +354,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if w["T"] is None:
-        ctx_lens = synth.serving_mix_ctx_lens(args.seed + rank, w["batch"])
-    else:
-        ctx_lens = [w["T"]] * w["batch"]
+    rank_seed, ctx_lens = rank_workload(w, args.seed, rank)
     config = {"workload": args.workload, "batch": w["batch"], "n_q_heads": w["n_q"], "n_kv_heads": w["n_kv"],
               "head_dim": w["d"], "ctx_len": w["T"] if w["T"] is not None else ctx_lens, "chunk_len": w["C"],
               "n_retain": w["n_retain"], "kv_budget": w.get("kv_budget", 0), "budget_frac": w.get("budget_frac", 0.0),
@@ -369,11 +392,11 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
 
-    inp = synth.make_chunk_inputs(args.seed + rank, w["batch"], w["n_q"], w["n_kv"], w["d"], ctx_lens, w["C"],
+    inp = synth.make_chunk_inputs(rank_seed, w["batch"], w["n_q"], w["n_kv"], w["d"], ctx_lens, w["C"],
                                   w["dtype"])
     paged = bool(w.get("paged"))
     if paged:
-        inp = synth.to_paged(inp, args.seed + rank)
+        inp = synth.to_paged(inp, rank_seed)
     q = inp.q.to(dev)
     k = (inp.k_pages if paged else inp.k).to(dev)
     v = (inp.v_pages if paged else inp.v).to(dev)
@@ -425,13 +448,8 @@ def main():
     launches = api.quoka_launch_count() - n0
     clocks = sampler.stop()
     dev_status = api.quoka_last_device_status(ws)
-    total_us = sum(per_step)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_us], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_us = float(t.item())
-    us_per_chunk = total_us / (args.steps * world)       # chunks processed by all ranks / time
+    total_us = max_over_ranks(sum(per_step), world, dev)
+    us_per_chunk = job_us_per_chunk(total_us, args.steps, world)
 
     if args.fused_only:
         if rank == 0:
@@ -507,13 +525,8 @@ def main():
             api.quoka_prefill_chunk_host(p, ctx_host, qh, knew, vnew, outh, q_dev, k, v, out, ws)
 
         ts = time_loop(e2e_step, args.steps, args.warmup, flush)
-        tot = sum(ts)
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([tot], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            tot = float(t.item())
-        e2e = {"value": round(tot / (args.steps * world), 2), "unit": UNIT,
+        tot = max_over_ranks(sum(ts), world, dev)
+        e2e = {"value": round(job_us_per_chunk(tot, args.steps, world), 2), "unit": UNIT,
                "h2d_bytes_per_step": qh.numel() * qh.element_size() + 2 * knew.numel() * knew.element_size(),
                "d2h_bytes_per_step": outh.numel() * outh.element_size()}
     else:
