@@ -343,6 +343,8 @@ def main():
     ap.add_argument("--fused-only", action="store_true",
                     help="only the timed fused steps (for profiler captures): no per-kernel, e2e or CPU legs")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--cached-norms", action="store_true",
+                    help="keep 1/|k| of every cache row beside the cache (quoka_update_key_norms) and let scoring read it")
     ap.add_argument("--sweep", action="store_true",
                     help="chunked prefill of the whole prompt (Algorithm 2): chunks at cached lengths 0, C, 2C, .. T, "
                          "eager launches and one CUDA graph, against the dense chunk kernel; prints its own JSON line")
@@ -407,6 +409,12 @@ def main():
     p = api.make_params(q, k, out, ctx, n_retain=w["n_retain"], kv_budget=w.get("kv_budget", 0),
                         budget_frac=w.get("budget_frac", 0.0), max_ctx_len=max(ctx_lens), block_table=bt, impl=impl)
     ws = api.alloc_workspace(p)
+    k_inv_norm = None
+    if args.cached_norms:
+        k_inv_norm = torch.zeros(tuple(k.shape[:3]), dtype=torch.float32, device=dev)
+        api.quoka_update_key_norms(p, k, k_inv_norm, True, ws)
+        p.k_inv_norm = k_inv_norm.data_ptr()
+        config["cached_key_norms"] = True
     cap = api.quoka_kv_budget_cap(p)
     b, n_q, C, d = q.shape
     n_kv = k.shape[1]

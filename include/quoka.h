@@ -105,6 +105,10 @@ typedef struct {
                                   number of pages in the pool when paged                        */
   int32_t score_mode;          /* quoka_score_mode; affects qbar (normalised or raw) and the scores */
   int32_t query_agg;           /* quoka_query_agg                                                 */
+  const float* k_inv_norm;     /* DEVICE, may be NULL: 1/max(|k|,1e-12) of every cache row, kept by the caller with
+                                  quoka_update_key_norms.  Indexed like the cache without head_dim: contiguous
+                                  [b][n_KV][kv_rows], paged [page][n_KV][64].  When given, quoka_score_keys and
+                                  quoka_prefill_chunk read it instead of recomputing the norms of all T_s keys  */
 } quoka_params;
 
 /* Row pitch of k_idx: the largest B_s any sequence can have, from max_ctx_len. */
@@ -134,6 +138,15 @@ quoka_status quoka_select_queries(const quoka_params* p, const void* q, int32_t*
  *   scores out [b][n_KV][max_ctx_len] fp32; entries t >= T_s are not written */
 quoka_status quoka_score_keys(const quoka_params* p, const void* qbar, const void* k_cache, float* scores,
                               void* ws, size_t ws_bytes, void* stream);
+
+/* Alg. 1 normalises every cached key in every chunk ("K <- K / norm(K)"); a cached key never changes, so its
+ * inverse norm can be computed once, when the key is appended, and kept beside the cache (the cost the paper's
+ * conclusion names as what is left to reduce is this pass over all T keys).  Writes
+ * k_inv_norm[row] = 1 / max(|k_row|, 1e-12) for rows [T_s, T_s + C) of every (sequence, KV head) (the chunk just
+ * appended), or for rows [0, T_s + C) when all_rows is non-zero (first use on an existing cache).
+ * p->k_inv_norm is ignored here; the output pointer is the argument. */
+quoka_status quoka_update_key_norms(const quoka_params* p, const void* k_cache, float* k_inv_norm, int32_t all_rows,
+                                    void* ws, size_t ws_bytes, void* stream);
 
 /* Alg. 1, I = topk(S^, B_SA) per (sequence, KV head): the B_s rows with the
  * largest score; among equal scores at the threshold the lower row wins; the

@@ -134,7 +134,14 @@ def aggregate_queries(q, q_idx, n_kv, storage="f32", score_mode="cosine"):
     return qbar
 
 
-def score_keys(qbar, k, T, score_mode="cosine", query_agg="max"):
+def key_inv_norms(k):
+    """1 / max(|k_t|, EPS) for every cache row.  Alg. 1 recomputes the key norms in every chunk; a caller may
+    keep these instead (a cached key never changes).  k: (n_KV, rows, d) -> (n_KV, rows)."""
+    k = np.asarray(k, dtype=np.float64)
+    return 1.0 / np.maximum(np.sqrt((k * k).sum(axis=2)), EPS)
+
+
+def score_keys(qbar, k, T, score_mode="cosine", query_agg="max", k_inv_norm=None):
     """K <- K / norm(K); S <- Q-bar K^T; S-hat <- max(S, dim=queries).
     qbar: (n_KV, N, d); k: (n_KV, >=T, d).  Returns (n_KV, T).
     The two ablations of the Appendix "Ablations": score_mode == "dot" leaves
@@ -143,7 +150,9 @@ def score_keys(qbar, k, T, score_mode="cosine", query_agg="max"):
     assert score_mode in ("cosine", "dot") and query_agg in ("max", "mean")
     qbar = np.asarray(qbar, dtype=np.float64)
     kc = np.asarray(k, dtype=np.float64)[:, :T, :]
-    if score_mode == "cosine":
+    if score_mode == "cosine" and k_inv_norm is not None:
+        k_hat = kc * np.asarray(k_inv_norm, dtype=np.float64)[:, :T, None]     # cached 1/|k| instead of a fresh norm
+    elif score_mode == "cosine":
         kn = np.maximum(np.sqrt((kc * kc).sum(axis=2, keepdims=True)), EPS)
         k_hat = kc / kn
     else:

@@ -24,7 +24,7 @@ AGG_MAX, AGG_MEAN = 0, 1
 
 EXPORTS = [
     "quoka_kv_budget_cap", "quoka_workspace_size", "quoka_select_queries", "quoka_score_keys",
-    "quoka_select_keys", "quoka_sparse_attn", "quoka_dense_chunk_attn", "quoka_prefill_chunk",
+    "quoka_update_key_norms", "quoka_select_keys", "quoka_sparse_attn", "quoka_dense_chunk_attn", "quoka_prefill_chunk",
     "quoka_prefill_chunk_host", "quoka_prefill_chunk_static", "quoka_last_device_status", "quoka_status_string", "quoka_launch_count",
 ]
 
@@ -47,6 +47,7 @@ class QuokaParams(C.Structure):
         ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_t", C.c_int64),
         ("kv_rows", C.c_int64),
         ("score_mode", C.c_int32), ("query_agg", C.c_int32),
+        ("k_inv_norm", C.c_void_p),
     ]
 
 
@@ -70,6 +71,7 @@ def load():
     lib.quoka_select_queries.argtypes = [pp, vp, vp, vp, vp, sz, vp]
     lib.quoka_score_keys.argtypes = [pp, vp, vp, vp, vp, sz, vp]
     lib.quoka_select_keys.argtypes = [pp, vp, vp, vp, vp, sz, vp]
+    lib.quoka_update_key_norms.argtypes = [pp, vp, vp, C.c_int32, vp, sz, vp]
     lib.quoka_sparse_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.quoka_dense_chunk_attn.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.quoka_prefill_chunk.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -159,6 +161,11 @@ def quoka_select_queries(p, q, q_idx, qbar, ws, stream=None):
 def quoka_score_keys(p, qbar, k_cache, scores, ws, stream=None):
     _check(load().quoka_score_keys(C.byref(p), _ptr(qbar), _ptr(k_cache), _ptr(scores), _ptr(ws), ws.numel(),
                                    _stream(stream)), "quoka_score_keys")
+
+
+def quoka_update_key_norms(p, k_cache, k_inv_norm, all_rows, ws, stream=None):
+    _check(load().quoka_update_key_norms(C.byref(p), _ptr(k_cache), _ptr(k_inv_norm), int(bool(all_rows)), _ptr(ws),
+                                         ws.numel(), _stream(stream)), "quoka_update_key_norms")
 
 
 def quoka_select_keys(p, scores, k_idx, k_cnt, ws, stream=None):

@@ -32,6 +32,8 @@ struct DevParams {
   int32_t* status;  // device status word
   int score_dot;    // 1: raw dot products (no normalisation of queries or keys)
   int agg_mean;     // 1: mean over the retained queries instead of the maximum
+  const float* k_inv_norm;  // cached 1/|k| per cache row, or null
+  int64_t kv_rows;  // rows per (sequence, head) when contiguous
 };
 
 // B_s of one sequence: min(B_SA, T) or floor(frac*T + 0.5) in double.
@@ -47,6 +49,13 @@ __device__ __forceinline__ int64_t kv_row_offset(const DevParams& P, int s, int 
   if (P.page_size == 0) return (int64_t)s * P.kv_sb + (int64_t)h * P.kv_sh + (int64_t)t * P.kv_st;
   const int page = __ldg(P.block_table + (int64_t)s * P.max_pages + (t >> 6));
   return (int64_t)page * P.kv_sb + (int64_t)h * P.kv_sh + (int64_t)(t & (kPage - 1)) * P.kv_st;
+}
+
+// Index of row t of (sequence s, KV head h) in the cached inverse-norm array (the cache's layout without head_dim).
+__device__ __forceinline__ int64_t kv_norm_index(const DevParams& P, int s, int h, int t) {
+  if (P.page_size == 0) return ((int64_t)s * P.n_kv + h) * P.kv_rows + t;
+  const int page = __ldg(P.block_table + (int64_t)s * P.max_pages + (t >> 6));
+  return ((int64_t)page * P.n_kv + h) * kPage + (t & (kPage - 1));
 }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
@@ -133,6 +142,8 @@ cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* 
                                      cudaStream_t st);
 cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,
                                    cudaStream_t st);
+cudaError_t launch_key_norms(const DevParams& P, int dtype, const void* k, float* k_inv_norm, int all_rows,
+                             cudaStream_t st);
 cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt,
                                cudaStream_t st);
 cudaError_t launch_attn_simt(const DevParams& P, int dtype, const void* q, const void* k, const void* v,

@@ -104,6 +104,8 @@ static DevParams make_dev(const quoka_params* p, void* ws) {
   P.status = static_cast<int32_t*>(ws);
   P.score_dot = p->score_mode == QUOKA_SCORE_DOT ? 1 : 0;
   P.agg_mean = p->query_agg == QUOKA_AGG_MEAN ? 1 : 0;
+  P.k_inv_norm = p->k_inv_norm;
+  P.kv_rows = p->kv_rows;
   return P;
 }
 
@@ -179,6 +181,17 @@ quoka_status quoka_score_keys(const quoka_params* p, const void* qbar, const voi
   if (!qbar || !k_cache || !scores || !aligned16(qbar) || !aligned16(k_cache)) return QUOKA_ERR_INVALID_ARG;
   if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
   return run_score_keys(p, make_dev(p, ws), qbar, k_cache, scores, static_cast<cudaStream_t>(stream));
+}
+
+quoka_status quoka_update_key_norms(const quoka_params* p, const void* k_cache, float* k_inv_norm, int32_t all_rows,
+                                    void* ws, size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!k_cache || !k_inv_norm || !aligned16(k_cache)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  QUOKA_TRY_CUDA(launch_key_norms(make_dev(p, ws), p->dtype, k_cache, k_inv_norm, all_rows ? 1 : 0,
+                                  static_cast<cudaStream_t>(stream)));
+  return QUOKA_OK;
 }
 
 quoka_status quoka_select_keys(const quoka_params* p, const float* scores, int32_t* k_idx, int32_t* k_cnt, void* ws,

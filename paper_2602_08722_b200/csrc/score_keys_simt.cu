@@ -66,8 +66,56 @@ __global__ void __launch_bounds__(kScoreTile) score_keys_simt_kernel(DevParams P
       if (j < nq) { best = fmaxf(best, acc[j]); total += acc[j]; }
   }
   if (t0 + tid < T)
-    scores[((int64_t)s * P.n_kv + kv) * P.max_ctx + t0 + tid] =
-        (P.agg_mean ? total / (float)N : best) / (P.score_dot ? 1.f : fmaxf(sqrtf(nn), kNormEps));
+  {
+    const float agg = P.agg_mean ? total / (float)N : best;
+    float val;
+    if (P.score_dot) val = agg;
+    else if (P.k_inv_norm) val = agg * __ldg(P.k_inv_norm + kv_norm_index(P, s, kv, t0 + tid));
+    else val = agg / fmaxf(sqrtf(nn), kNormEps);
+    scores[((int64_t)s * P.n_kv + kv) * P.max_ctx + t0 + tid] = val;
+  }
+}
+
+// Inverse norms of cache rows (one warp per row): rows [T_s, T_s + C) of every (sequence, KV head), or all of
+// [0, T_s + C).  HBM-bound: one read of the rows.
+template <typename E, int D>
+__global__ void __launch_bounds__(256) key_norms_kernel(DevParams P, const E* __restrict__ k, float* __restrict__ out,
+                                                         int all_rows, int rows_max) {
+  constexpr int NE = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int r = (int)(warp % rows_max);
+  const int kv = (int)((warp / rows_max) % P.n_kv);
+  const int s = (int)(warp / ((int64_t)rows_max * P.n_kv));
+  if (s >= P.batch) return;
+  const int T = __ldg(P.ctx_len + s);
+  const int first = all_rows ? 0 : T, count = all_rows ? T + P.chunk : P.chunk;
+  if (r >= count) return;
+  const int t = first + r;
+  float x[NE];
+  load_vec<E, NE>(k + kv_row_offset(P, s, kv, t) + lane * NE, x);
+  float nn = 0.f;
+#pragma unroll
+  for (int i = 0; i < NE; ++i) nn = fmaf(x[i], x[i], nn);
+  nn = warp_sum(nn);
+  if (lane == 0) out[kv_norm_index(P, s, kv, t)] = 1.f / fmaxf(sqrtf(nn), kNormEps);
+}
+
+cudaError_t launch_key_norms(const DevParams& P, int dtype, const void* k, float* k_inv_norm, int all_rows,
+                             cudaStream_t st) {
+  const int rows_max = all_rows ? P.max_ctx + P.chunk : P.chunk;
+  const int64_t warps = (int64_t)P.batch * P.n_kv * rows_max;
+  const int grid = (int)((warps * 32 + 255) / 256);
+  if (grid <= 0) return cudaSuccess;
+  if (dtype == QUOKA_BF16) {
+    if (P.d == 128) key_norms_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16*)k, k_inv_norm, all_rows, rows_max);
+    else key_norms_kernel<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16*)k, k_inv_norm, all_rows, rows_max);
+  } else {
+    if (P.d == 128) key_norms_kernel<float, 128><<<grid, 256, 0, st>>>(P, (const float*)k, k_inv_norm, all_rows, rows_max);
+    else key_norms_kernel<float, 64><<<grid, 256, 0, st>>>(P, (const float*)k, k_inv_norm, all_rows, rows_max);
+  }
+  count_launch();
+  return cudaGetLastError();
 }
 
 cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,

@@ -229,9 +229,17 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
       slot = slots == 2 ? group : 0;
       acc_phase = slots == 2 ? (uint32_t)((n_done >> 1) & 1) : (uint32_t)(n_done & 1);
       if (!mbar_wait(&full[stage], phase, wc)) break;
-      // |k|^2 from the tile in shared memory (rotated 16-byte reads: conflict-free)
+      // 1/|k|: read from the caller's cache of inverse norms when there is one (the load is in flight under the
+      // accumulator wait), else |k|^2 from the tile in shared memory (rotated 16-byte reads: conflict-free)
+      const int T_s = __ldg(P.ctx_len + w.s);
+      const int t = w.tile * kTileKeys + row;
+      const bool own_norm = P.k_inv_norm == nullptr && !P.score_dot;
+      float inv_cached = 1.f;
+      if (P.k_inv_norm != nullptr && !P.score_dot)
+        inv_cached = __ldg(P.k_inv_norm + kv_norm_index(P, w.s, w.kv, min(t, T_s - 1)));
       float nacc[4] = {0.f, 0.f, 0.f, 0.f};                 // independent partial sums: no 256-deep FMA chain
       const unsigned char* krow = k_smem + (size_t)stage * kStageBytes + row * 128;
+      if (own_norm) {
 #pragma unroll
       for (int h = 0; h < HALVES; ++h) {
 #pragma unroll
@@ -245,6 +253,7 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
             nacc[i] = fmaf(b, b, nacc[i]);
           }
         }
+      }
       }
       const float nn = (nacc[0] + nacc[1]) + (nacc[2] + nacc[3]);
       __syncwarp();
@@ -311,9 +320,9 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[slot]);
-      const int t = w.tile * kTileKeys + row;
-      if (t < __ldg(P.ctx_len + w.s))
-        scores[((long long)w.s * P.n_kv + w.kv) * P.max_ctx + t] = P.score_dot ? best : best / fmaxf(sqrtf(nn), kNormEps);
+      if (t < T_s)
+        scores[((long long)w.s * P.n_kv + w.kv) * P.max_ctx + t] =
+            own_norm ? best / fmaxf(sqrtf(nn), kNormEps) : best * inv_cached;
       if (++stage == A.stages) { stage = 0; phase ^= 1; }
     }
   }

@@ -96,7 +96,7 @@ class GpuProblem:
     """Device buffers + params for one ChunkInputs."""
 
     def __init__(self, inp, n_retain, kv_budget=0, budget_frac=0.0, impl=api.IMPL_AUTO, paged=False,
-                 max_ctx_len=None, score_mode="cosine", query_agg="max"):
+                 max_ctx_len=None, score_mode="cosine", query_agg="max", cached_norms=False):
         dev = "cuda"
         self.inp = inp
         self.dtype = inp.dtype
@@ -130,6 +130,12 @@ class GpuProblem:
         self.k_idx = torch.full((b, n_kv, self.cap), -7, dtype=torch.int32, device=dev)
         self.k_cnt = torch.full((b,), -7, dtype=torch.int32, device=dev)
         self.lse = torch.zeros((b, n_q, C), dtype=torch.float32, device=dev)
+        self.k_inv_norm = None
+        if cached_norms:
+            # the cache of inverse key norms: built once for the rows already there, then kept per appended chunk
+            self.k_inv_norm = torch.full(tuple(self.k.shape[:3]), float("nan"), dtype=torch.float32, device=dev)
+            api.quoka_update_key_norms(self.p, self.k, self.k_inv_norm, True, self.ws)
+            self.p.k_inv_norm = self.k_inv_norm.data_ptr()
 
     def run_staged(self):
         api.quoka_select_queries(self.p, self.q, self.q_idx, self.qbar, self.ws)

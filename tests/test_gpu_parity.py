@@ -14,12 +14,12 @@ IMPLS = [pytest.param(api.IMPL_SIMT, id="simt"), pytest.param(api.IMPL_AUTO, id=
 
 def problem(seed, *, batch=1, n_q=4, n_kv=2, d=128, T=1000, C=300, dtype="bf16", n_retain=24, kv_budget=177,
             budget_frac=0.0, impl=api.IMPL_AUTO, paged=False, capacity=None, max_ctx_len=None, score_mode="cosine",
-            query_agg="max"):
+            query_agg="max", cached_norms=False):
     inp = synth.make_chunk_inputs(seed, batch, n_q, n_kv, d, T, C, dtype, capacity=capacity)
     if paged:
         inp = synth.to_paged(inp, seed)
     return GpuProblem(inp, n_retain, kv_budget, budget_frac, impl=impl, paged=paged, max_ctx_len=max_ctx_len,
-                      score_mode=score_mode, query_agg=query_agg)
+                      score_mode=score_mode, query_agg=query_agg, cached_norms=cached_norms)
 
 
 # ---------------------------------------------------------------- small cases, every stage, all rows
@@ -106,6 +106,38 @@ def test_decode_step_full_size_32k():
                  kv_budget=w["kv_budget"])
     gp.run_staged()
     check_chain(gp)
+
+
+# ---------------------------------------------------------------- cached inverse key norms
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("paged", [False, True])
+def test_cached_key_norms(paged, impl):
+    gp = problem(16, batch=2, n_q=8, n_kv=2, T=[1700, 640], C=200, n_retain=24, kv_budget=0, budget_frac=0.2, impl=impl,
+                 paged=paged, cached_norms=True)
+    # the cache itself against the oracle, on every row that exists
+    for s in range(gp.b):
+        T = int(gp.inp.ctx_len[s])
+        want = O.key_inv_norms(f64(gp.inp.k[s, :, : T + gp.C]))
+        if paged:
+            tbl = gp.inp.block_table[s]
+            got = np.stack([f64(gp.k_inv_norm[int(tbl[t // 64]), :, t % 64]) for t in range(T + gp.C)], axis=1)
+        else:
+            got = f64(gp.k_inv_norm[s, :, : T + gp.C])
+        np.testing.assert_allclose(got, want, rtol=2e-6)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(staged, gp.out)
+    # appending: only the chunk's rows are rewritten
+    before = gp.k_inv_norm.clone()
+    gp.k_inv_norm.fill_(7.0)
+    api.quoka_update_key_norms(gp.p, gp.k, gp.k_inv_norm, False, gp.ws)
+    torch.cuda.synchronize()
+    changed = gp.k_inv_norm != 7.0
+    assert int(changed.sum()) == gp.b * gp.n_kv * gp.C
+    assert torch.equal(gp.k_inv_norm[changed], before[changed])
 
 
 # ---------------------------------------------------------------- ablation variants of the scoring step

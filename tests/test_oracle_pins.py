@@ -132,6 +132,31 @@ def test_ablation_variants_hand_example_and_invariants():
     np.testing.assert_allclose(got, dots.max(axis=1), atol=1e-12)
 
 
+def test_cached_inverse_key_norms_hand_values_and_equivalence():
+    g = _load_golden()
+    k = g["k"].reshape(1, 4, 2)
+    # |k| = 3, 5, 2*sqrt(2), 2 for the hand example's keys
+    np.testing.assert_allclose(O.key_inv_norms(k)[0], [1 / 3, 0.2, 1 / (2 * np.sqrt(2)), 0.5], atol=1e-15)
+    q, kr, _ = rand_problem(6, n_q=4, n_kv=2, C=9, d=8, T=13)
+    idx, _ = O.select_queries(q, 3)
+    qb = O.aggregate_queries(q, idx, 2)
+    inv = O.key_inv_norms(kr)
+    np.testing.assert_allclose(inv, 1.0 / np.linalg.norm(kr, axis=2), rtol=1e-14)
+    for agg in ("max", "mean"):
+        np.testing.assert_allclose(O.score_keys(qb, kr, 13, "cosine", agg, k_inv_norm=inv),
+                                   O.score_keys(qb, kr, 13, "cosine", agg), atol=1e-14)
+    # the cache is used as given: a stale entry changes exactly that key's score, by the ratio
+    stale = inv.copy()
+    stale[:, 4] *= 2.0
+    a = O.score_keys(qb, kr, 13, k_inv_norm=stale)
+    b = O.score_keys(qb, kr, 13)
+    np.testing.assert_allclose(a[:, 4], 2.0 * b[:, 4], atol=1e-14)
+    np.testing.assert_allclose(np.delete(a, 4, axis=1), np.delete(b, 4, axis=1), atol=1e-14)
+    # dot-product scoring ignores it; a zero key gets the clamped inverse, not infinity
+    np.testing.assert_allclose(O.score_keys(qb, kr, 13, "dot", k_inv_norm=stale), O.score_keys(qb, kr, 13, "dot"), atol=0)
+    assert np.isfinite(O.key_inv_norms(np.zeros((1, 2, 4)))).all()
+
+
 # ------------------------------------------------------------------ query sub-selection
 def test_query_cosines_match_library_cosine_distance():
     q, _, _ = rand_problem(1, n_q=3, C=17, d=8)
@@ -450,6 +475,8 @@ MUTANTS = {
     "dot mode normalises keys": ("    else:\n        k_hat = kc", "    else:\n        k_hat = kc / np.sqrt((kc * kc).sum(axis=2, keepdims=True))"),
     "dot mode normalises queries": ("    else:\n        q_hat = gathered", "    else:\n        q_hat = gathered / np.sqrt((gathered * gathered).sum(axis=2, keepdims=True))"),
     "mean mode sums": ("else S.mean(axis=1)", "else S.sum(axis=1)"),
+    "cached norm used as a norm": ("k_hat = kc * np.asarray(k_inv_norm", "k_hat = kc / np.asarray(k_inv_norm"),
+    "inverse norm of the squared norm": ("return 1.0 / np.maximum(np.sqrt((k * k).sum(axis=2)), EPS)", "return 1.0 / np.maximum((k * k).sum(axis=2), EPS)"),
 }
 
 PIN_TESTS = [
@@ -463,6 +490,7 @@ PIN_TESTS = [
     test_identical_keys_give_uniform_average_of_visible_values,
     test_full_budget_and_all_queries_equals_dense, test_query_cosines_match_library_cosine_distance,
     test_selection_invariant_to_positive_rescaling, test_ablation_variants_hand_example_and_invariants,
+    test_cached_inverse_key_norms_hand_values_and_equivalence,
 ]
 
 
