@@ -165,24 +165,19 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       tc_fence_after();
       const int lim = visible_cols<SPARSE>(g, j, row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
-      // ---- pass 1: the row maximum, 32 columns at a time with the next load in flight.  The row is read
-      // once here and once more by pass 2: tensor memory is cheap to re-read, and not keeping 128 values
-      // live leaves pass 2 the registers it needs to keep a whole block of exponentials in flight.
+      // ---- pass 1: the row maximum.  All four 32-column loads are issued together (one tensor-memory round
+      // trip); the row is read once more, in 64-key blocks, by pass 2: tensor memory is cheap to re-read, and
+      // not keeping the 128 values live leaves pass 2 the registers for a whole block of exponentials in flight.
       float mx;
       {
-        uint32_t c0[32], c1[32];
+        uint32_t c0[32], c1[32], c2[32], c3[32];
         tmem_ld32(s_addr, c0);
-        tmem_wait_ld();
         tmem_ld32(s_addr + 32, c1);
-        mx = max32(c0, masked, 0, lim);
+        tmem_ld32(s_addr + 64, c2);
+        tmem_ld32(s_addr + 96, c3);
         tmem_wait_ld();
-        tmem_ld32(s_addr + 64, c0);
-        mx = fmaxf(mx, max32(c1, masked, 32, lim));
-        tmem_wait_ld();
-        tmem_ld32(s_addr + 96, c1);
-        mx = fmaxf(mx, max32(c0, masked, 64, lim));
-        tmem_wait_ld();
-        mx = fmaxf(mx, max32(c1, masked, 96, lim));
+        mx = fmaxf(fmaxf(max32(c0, masked, 0, lim), max32(c1, masked, 32, lim)),
+                   fmaxf(max32(c2, masked, 64, lim), max32(c3, masked, 96, lim)));
       }
       const float m_tile = mx * scale_log2;
       // ---- lazy rescale of the accumulator: only when some row's maximum grew by more than the threshold

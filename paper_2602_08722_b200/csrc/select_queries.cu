@@ -14,6 +14,8 @@
 //                their j-th retained query, each divided by its own norm; one rounding to dtype.
 #include <cooperative_groups.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace cg = cooperative_groups;
@@ -46,14 +48,14 @@ __device__ __forceinline__ void raw_to_f32(const Raw8<T>& r, float (&x)[8]) {
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P, const T* __restrict__ q,
+__global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams P, const T* __restrict__ q,
                                                                      int32_t* __restrict__ q_idx, int rpc, int n_sort,
                                                                      int staged, int m_peer) {
   constexpr int LG = D / 8;                 // lanes per row, 8 elements each
   constexpr int RPI = kRankThreads / LG;    // rows per iteration
   constexpr int NW = sizeof(T) * 8 / 16;    // 16-byte words per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // dynamic shared memory: sort keys | reduction buffer | row norms | staged rows
+  // dynamic shared memory: sort keys | reduction buffer | (unused) | peer codes | staged rows
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);               // [n_sort] 32-key sorted runs
   unsigned long long* sorted = keys + n_sort;                                               // [n_sort] the sorted slice
   float* red = reinterpret_cast<float*>(smem_raw + (size_t)n_sort * 16);                    // [RPI][D]
@@ -61,7 +63,7 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   unsigned long long* peer_keys = reinterpret_cast<unsigned long long*>(norms + ((rpc + 3) & ~3));   // [7][m_peer]
   uint4* rows = reinterpret_cast<uint4*>(peer_keys + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1));   // [rpc][LG][NW]
   __shared__ float part[D];                 // this CTA's share of the column sums
-  __shared__ float M[D];
+  __shared__ __align__(16) float M[D];
   __shared__ float Mnorm;
 
   cg::cluster_group cluster = cg::this_cluster();
@@ -84,8 +86,8 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   const int n_loc = hi - lo;
 
   // ---- pass 1: the slice goes to shared memory with every 16-byte copy in flight at once, committed in 8
-  // groups of rows; column sums and row norms are taken group by group as the copies land, so the arithmetic
-  // runs under the HBM transfer
+  // groups of rows; the column sums are taken group by group as the copies land, so the arithmetic runs under
+  // the HBM transfer
   const int n_iter = (n_loc + RPI - 1) / RPI;                // 32/64-row trips over the slice
   const int grp_rows = ((n_iter + 7) / 8) * RPI;             // rows per copy group
   if (staged) {
@@ -98,7 +100,8 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
       for (int w = w_lo + tid; w < w_hi; w += kRankThreads) {
         const int r = w / WPR, c = w % WPR;
         const T* src = qh + (long long)(lo + r) * P.q_st + c * EPW;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(rows_s + (uint32_t)w * 16u), "l"(src) : "memory");
+        // word c of row r lives in slot c ^ (r & 7): both passes then read shared memory without bank conflicts
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(rows_s + (uint32_t)(r * WPR + (c ^ (r & 7))) * 16u), "l"(src) : "memory");
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
@@ -122,14 +125,13 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
       __syncthreads();
     }
     const int g_lo = min(n_loc, gi * grp_rows), g_hi = min(n_loc, (gi + 1) * grp_rows);
-    for (int r0 = g_lo; r0 < g_hi; r0 += RPI) {              // uniform trip count: the shuffles below need whole warps
+    for (int r0 = g_lo; r0 < g_hi; r0 += RPI) {
       const int r = r0 + row_slot;
-      float nn = 0.f;
       Raw8<T> raw;
       const int rc = min(r, n_loc - 1);                      // clamped: no branch around the loads
       if (staged) {
 #pragma unroll
-        for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)rc * LG + lane_in_row) * NW + w];
+        for (int w = 0; w < NW; ++w) raw.w[w] = rows[(size_t)rc * (LG * NW) + ((lane_in_row * NW + w) ^ (rc & 7))];
       } else {
         const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)(lo + rc) * P.q_st + lane_in_row * 8);
 #pragma unroll
@@ -139,10 +141,7 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
       raw_to_f32<T>(raw, x);
       const float live = r < n_loc ? 1.f : 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { acc[i] = fmaf(x[i], live, acc[i]); nn = fmaf(x[i], x[i], nn); }
-#pragma unroll
-      for (int o = LG / 2; o > 0; o >>= 1) nn += __shfl_xor_sync(0xFFFFFFFFu, nn, o);
-      if (lane_in_row == 0 && r < n_loc) norms[r] = fmaxf(sqrtf(nn), kNormEps);
+      for (int i = 0; i < 8; ++i) acc[i] = fmaf(x[i], live, acc[i]);
     }
   }
 #pragma unroll
@@ -169,38 +168,57 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   }
   __syncthreads();
 
-  // ---- pass 2: cosine of every row of the slice to M, packed as (order code << 32 | position)
-  float m[8];
+  // ---- pass 2: cosine of every row of the slice to M, packed as (order code << 32 | position).  Two adjacent
+  // lanes take one row (half of its 16-byte words each, the row's norm and its dot product with M in the same
+  // sweep, M read from shared memory as a broadcast); one shuffle joins the halves.
+  {
+    constexpr int WPR = LG * NW;                             // 16-byte words per row
+    constexpr int EPW = 16 / (int)sizeof(T);                 // elements per word
+    constexpr int HW = WPR / 2;                              // words per half row
+    const int half = tid & 1;
+    const float mn = Mnorm;
+    auto sweep = [&](auto from_smem) {                       // the staged / re-read choice is made once, not per word
+    for (int r0 = 0; r0 < n_sort; r0 += kRankThreads / 2) {
+      const int r = r0 + (tid >> 1);
+      const int rc = max(min(r, n_loc - 1), 0);              // clamped (an empty slice reads row 0 / the last row)
+      const uint4* grow = reinterpret_cast<const uint4*>(qh + (long long)min(lo + rc, C - 1) * P.q_st);
+      float dot = 0.f, nn = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) m[i] = M[lane_in_row * 8 + i];
-  const float mn = Mnorm;
-  for (int r0 = 0; r0 < n_sort; r0 += RPI) {
-    const int r = r0 + row_slot;
-    const int rc = max(min(r, n_loc - 1), 0);             // clamped (an empty slice reads row 0 / the last row)
-    Raw8<T> raw;
-    if (staged) {
+      for (int i = 0; i < HW; ++i) {
+        const int c = half * HW + i;
+        uint4 wv;
+        if constexpr (decltype(from_smem)::value) wv = rows[(size_t)rc * WPR + (c ^ (rc & 7))];
+        else wv = __ldg(grow + c);
+        float x[EPW];
+        if constexpr (sizeof(T) == 2) {
+          const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
-      for (int w = 0; w < NW; ++w) raw.w[w] = rows[((size_t)rc * LG + lane_in_row) * NW + w];
-    } else {
-      const uint4* src = reinterpret_cast<const uint4*>(qh + (long long)min(lo + rc, C - 1) * P.q_st + lane_in_row * 8);
+          for (int j = 0; j < 4; ++j) { x[2 * j] = __uint_as_float(ww[j] << 16); x[2 * j + 1] = __uint_as_float(ww[j] & 0xFFFF0000u); }
+        } else {
+          x[0] = __uint_as_float(wv.x); x[1] = __uint_as_float(wv.y); x[2] = __uint_as_float(wv.z); x[3] = __uint_as_float(wv.w);
+        }
 #pragma unroll
-      for (int w = 0; w < NW; ++w) raw.w[w] = __ldg(src + w);
-    }
-    float x[8];
-    raw_to_f32<T>(raw, x);
-    float dot = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) dot = fmaf(x[i], m[i], dot);
-#pragma unroll
-    for (int o = LG / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
-    if (lane_in_row == 0 && r < n_sort) {
-      unsigned long long code = ~0ull;                    // padding sorts last
-      if (r < n_loc) {
-        const float c = dot / (norms[r] * mn);
-        code = ((unsigned long long)float_order_key(c) << 32) | (unsigned)(lo + r);
+        for (int j = 0; j < EPW; j += 4) {
+          const float4 mv = *reinterpret_cast<const float4*>(&M[c * EPW + j]);
+          dot = fmaf(x[j], mv.x, dot); dot = fmaf(x[j + 1], mv.y, dot);
+          dot = fmaf(x[j + 2], mv.z, dot); dot = fmaf(x[j + 3], mv.w, dot);
+          nn = fmaf(x[j], x[j], nn); nn = fmaf(x[j + 1], x[j + 1], nn);
+          nn = fmaf(x[j + 2], x[j + 2], nn); nn = fmaf(x[j + 3], x[j + 3], nn);
+        }
       }
-      keys[r] = code;
+      dot += __shfl_xor_sync(0xFFFFFFFFu, dot, 1);
+      nn += __shfl_xor_sync(0xFFFFFFFFu, nn, 1);
+      if (half == 0 && r < n_sort) {
+        unsigned long long code = ~0ull;                    // padding sorts last
+        if (r < n_loc) {
+          const float c = dot / (fmaxf(sqrtf(nn), kNormEps) * mn);
+          code = ((unsigned long long)float_order_key(c) << 32) | (unsigned)(lo + r);
+        }
+        keys[r] = code;
+      }
     }
+    };
+    if (staged) sweep(std::true_type{}); else sweep(std::false_type{});
   }
   __syncthreads();
 
@@ -230,13 +248,24 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
     const int my_run = i >> 5;
     int rk = i & 31;
 #pragma unroll 1
-    for (int run = 0; run < n_runs; ++run) {
-      const unsigned long long* pr = keys + run * 32;
-      int pos = 0;
+    for (int run0 = 0; run0 < n_runs; run0 += 8) {        // eight searches side by side: their loads overlap
+      int pos[8];
 #pragma unroll
-      for (int step = 16; step > 0; step >>= 1) pos += pr[pos + step - 1] < key ? step : 0;
-      pos += pr[pos] < key ? 1 : 0;
-      rk += run == my_run ? 0 : pos;
+      for (int u = 0; u < 8; ++u) pos[u] = 0;
+#pragma unroll
+      for (int step = 16; step > 0; step >>= 1) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int run = min(run0 + u, n_runs - 1);
+          pos[u] += keys[run * 32 + pos[u] + step - 1] < key ? step : 0;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int run = min(run0 + u, n_runs - 1);
+        pos[u] += keys[run * 32 + pos[u]] < key ? 1 : 0;
+        rk += (run0 + u < n_runs && run != my_run) ? pos[u] : 0;
+      }
     }
     sorted[rk] = key;                                     // padding keys are equal: they may collide, all ~0
   }
@@ -256,13 +285,18 @@ __global__ void __launch_bounds__(kRankThreads) rank_queries_kernel(DevParams P,
   for (int li = tid; li < n_cand; li += kRankThreads) {
     const unsigned long long key = sorted[li];
     int rk = li;
-#pragma unroll 1
+    int pos[kRankCluster - 1];                            // number of each peer's codes below key; the seven
+#pragma unroll                                            // branch-free searches run side by side
+    for (int pr = 0; pr < kRankCluster - 1; ++pr) pos[pr] = 0;
+    for (int step = m_peer >> 1; step > 0; step >>= 1) {
+#pragma unroll
+      for (int pr = 0; pr < kRankCluster - 1; ++pr)
+        pos[pr] += peer_keys[(size_t)pr * m_peer + pos[pr] + step - 1] < key ? step : 0;
+    }
+#pragma unroll
     for (int pr = 0; pr < kRankCluster - 1; ++pr) {
-      const unsigned long long* pk = peer_keys + (size_t)pr * m_peer;
-      int pos = 0;                                        // number of pk[] entries below key, branch-free
-      for (int step = m_peer >> 1; step > 0; step >>= 1) pos += pk[pos + step - 1] < key ? step : 0;
-      pos += pk[pos] < key ? 1 : 0;
-      rk += pos;
+      pos[pr] += peer_keys[(size_t)pr * m_peer + pos[pr]] < key ? 1 : 0;
+      rk += pos[pr];
     }
     if (rk < N) out[rk] = (int32_t)(key & 0xFFFFFFFFull);
   }
