@@ -44,43 +44,102 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Every CTA walks ONE sequence of key tiles t = 0 .. n_total-1 for both of its Q tiles; Q tile x takes part in
+// the tiles t >= skip[x] (a suffix, so both finish on the same tile).
+//   dense : the tiles of rows [0, T + C) in DESCENDING order (the tiles only Q tile B sees come first).
+//   sparse: first the chunk's own tiles (the one only B sees, then tiles 0 .. c_a-1), THEN the tiles of the
+//           selected list.  The chunk's tiles do not depend on the key selection, so this kernel is launched
+//           with programmatic stream serialisation: it starts while the selection kernel still runs, works
+//           through the chunk tiles, and only then waits for the selection (`resolve`) to learn the list length.
 struct AttnGeom {
-  int T, cnt, n_sel;        // cached length, selected rows, selected tiles (sparse); cnt = T, n_sel unused (dense)
-  int n_a, n_b, n_max;      // key tiles Q tile A / B take part in, and their maximum
+  int T, C;
+  int n_chunk;        // sparse: tiles of the chunk's own rows in the sequence; dense: 0
+  int c_a;            // sparse: chunk tiles Q tile A sees
+  int b_first;        // sparse: 1 when the sequence starts with the tile only B sees
+  int skip_a;         // first tile Q tile A takes part in (B takes part in all); scalars, not arrays: the struct
+  bool active_b;      // must live in registers (an indexed member would put it in local memory)
+  int n_known;        // tiles known so far (sparse: n_chunk until resolved, then n_chunk + n_sel)
+  int cnt;            // sparse: selected rows (valid once resolved)
+  int n_dense;        // dense: number of tiles
+  bool resolved;
 };
 
 template <bool SPARSE>
-__device__ __forceinline__ AttnGeom make_geom(const DevParams& P, int s, int r0, const int32_t* k_cnt) {
+__device__ __forceinline__ AttnGeom make_geom(const DevParams& P, int s, int r0) {
   AttnGeom g;
   g.T = __ldg(P.ctx_len + s);
-  const int C = P.chunk;
-  const bool b_active = r0 + kQTile < C;
+  g.C = P.chunk;
+  const bool b_active = r0 + kQTile < g.C;
+  g.active_b = b_active;
+  g.cnt = 0;
   if (SPARSE) {
-    g.cnt = __ldg(k_cnt + s);
-    g.n_sel = (g.cnt + kKeyTile - 1) / kKeyTile;
-    g.n_a = g.n_sel + r0 / kQTile + 1;
-    g.n_b = b_active ? g.n_a + 1 : 0;
+    g.c_a = r0 / kQTile + 1;
+    g.b_first = b_active ? 1 : 0;
+    g.n_chunk = g.c_a + g.b_first;
+    g.skip_a = g.b_first;
+    g.n_known = g.n_chunk;
+    g.n_dense = 0;
+    g.resolved = false;
   } else {
-    g.cnt = g.T;
-    g.n_sel = 0;
-    const int last_a = min(r0 + kQTile - 1, C - 1), last_b = min(r0 + 2 * kQTile - 1, C - 1);
-    g.n_a = (g.T + last_a) / kKeyTile + 1;
-    g.n_b = b_active ? (g.T + last_b) / kKeyTile + 1 : 0;
+    const int last_a = min(r0 + kQTile - 1, g.C - 1), last_b = min(r0 + 2 * kQTile - 1, g.C - 1);
+    const int n_a = (g.T + last_a) / kKeyTile + 1;
+    const int n_b = b_active ? (g.T + last_b) / kKeyTile + 1 : 0;
+    g.n_dense = max(n_a, n_b);
+    g.skip_a = g.n_dense - n_a;
+    g.n_chunk = 0; g.c_a = 0; g.b_first = 0;
+    g.n_known = g.n_dense;
+    g.resolved = true;
   }
-  g.n_max = max(g.n_a, g.n_b);
   return g;
 }
 
-// Number of visible columns of key tile j for chunk row `row` (columns [0, lim) are visible).
+// Sparse: wait for the selection kernel (a no-op when this kernel was not launched early) and read the list length.
+__device__ __forceinline__ void resolve(AttnGeom& g, const int32_t* k_cnt, int s) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  g.cnt = __ldcg(k_cnt + s);
+  g.n_known = g.n_chunk + (g.cnt + kKeyTile - 1) / kKeyTile;
+  g.resolved = true;
+}
+
+// Rows of tile t: from the selected list (`from_list`, rows list[base .. base + count)), or the consecutive cache
+// rows first .. first + count - 1.  `diag` = chunk position of the tile's first row minus one tile-relative
+// offset, used by the causal limit: row r sees columns [0, r - col0 + 1).
+struct TileRows {
+  bool from_list;
+  int first, count;     // consecutive rows (count may exceed the tile or be <= 0), or list base and remaining count
+  int col0;             // causal tiles: chunk position (dense: position in [0, T + C)) of column 0; list tiles: unused
+};
+
 template <bool SPARSE>
-__device__ __forceinline__ int visible_cols(const AttnGeom& g, int j, int row) {
-  int lim;
+__device__ __forceinline__ TileRows tile_rows(const AttnGeom& g, int t) {
+  TileRows r;
   if (SPARSE) {
-    if (j < g.n_sel) lim = g.cnt - j * kKeyTile;
-    else lim = row - (j - g.n_sel) * kKeyTile + 1;
+    if (t < g.n_chunk) {
+      const int ct = g.b_first ? (t == 0 ? g.c_a : t - 1) : t;
+      r.from_list = false;
+      r.first = g.T + ct * kKeyTile;
+      r.count = g.C - ct * kKeyTile;
+      r.col0 = ct * kKeyTile;
+    } else {
+      const int st = t - g.n_chunk;
+      r.from_list = true;
+      r.first = st * kKeyTile;
+      r.count = g.cnt - st * kKeyTile;
+      r.col0 = 0;
+    }
   } else {
-    lim = g.T + row - j * kKeyTile + 1;
+    const int j = g.n_dense - 1 - t;
+    r.from_list = false;
+    r.first = j * kKeyTile;
+    r.count = g.T + g.C - j * kKeyTile;
+    r.col0 = j * kKeyTile - g.T;            // chunk position of column 0 (negative inside the cache)
   }
+  return r;
+}
+
+// Number of visible columns of tile t for chunk row `row` (columns [0, lim) are visible).
+__device__ __forceinline__ int visible_cols(const TileRows& tr, int row) {
+  const int lim = tr.from_list ? tr.count : row - tr.col0 + 1;
   return max(0, min(kKeyTile, lim));
 }
 
@@ -129,7 +188,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
   const int s = blockIdx.z, h = blockIdx.x, kv = h / P.group;
   const int rb = gridDim.y - 1 - blockIdx.y;
   const int r0 = rb * 2 * kQTile;
-  const AttnGeom g = make_geom<SPARSE>(P, s, r0, k_cnt);
+  AttnGeom g = make_geom<SPARSE>(P, s, r0);
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -149,7 +208,6 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
   if (warp < 8) {
     // ================================================================== softmax + epilogue
     const int x = warp >> 2;                                  // Q tile A (0) or B (1)
-    const int n_tiles = x ? g.n_b : g.n_a;
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
     const int row = r0 + x * kQTile + row_in_tile;            // chunk row
@@ -159,11 +217,18 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     float m_run = -INFINITY, l_run = 0.f;
     uint32_t phase = 0;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
+    const int skip_x = x ? 0 : g.skip_a;
+    const bool active_x = x ? g.active_b : true;
+    for (int t = skip_x; active_x; ++t) {
+      if (t == g.n_known) {                                   // end of what is known: the list length, or the end
+        if (g.resolved) break;
+        resolve(g, k_cnt, s);
+        if (t == g.n_known) break;
+      }
       if (!mbar_wait(&s_full[x], phase, wc)) { ok = false; break; }
       phase ^= 1;
       tc_fence_after();
-      const int lim = visible_cols<SPARSE>(g, j, row);
+      const int lim = visible_cols(tile_rows<SPARSE>(g, t), row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
       // ---- pass 1: the row maximum.  All four 32-column loads are issued together (one tensor-memory round
       // trip); the row is read once more, in 64-key blocks, by pass 2: tensor memory is cheap to re-read, and
@@ -184,7 +249,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       const bool grow = m_tile > m_run + kRescaleThreshold;
       if (__any_sync(0xFFFFFFFFu, grow)) {
         const float m_new = fmaxf(m_run, m_tile);
-        if (j > 0) {
+        if (t > skip_x) {
           const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
           l_run *= alpha;
 #pragma unroll
@@ -237,7 +302,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       l_run += (ps0 + ps1) + (ps2 + ps3);
     }
     // ---- epilogue: O / l -> bf16 -> global
-    if (ok && n_tiles > 0 && mbar_wait(&o_full[x], 0, wc)) {
+    if (ok && active_x && mbar_wait(&o_full[x], 0, wc)) {
       tc_fence_after();
       const float inv = 1.f / l_run;
       const bool store = row < P.chunk;
@@ -276,7 +341,6 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     const int c16 = lane % PIECES;                            // this thread's piece of the row
     const int rsub = lane / PIECES;
     const int32_t* idx = SPARSE ? k_idx + ((long long)s * P.n_kv + kv) * P.budget_cap : nullptr;
-    const int n_items = 2 * g.n_max;
     uint32_t phase = 0;
     int slot = 0;
     const uint32_t kv_base = smem_u32(kv_smem);
@@ -286,67 +350,76 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     const uint32_t base16 = (uint32_t)(((P.page_size == 0 ? (long long)s * P.kv_sb : 0ll) + (long long)kv * P.kv_sh) >> 3) +
                             (uint32_t)c16;
     const int32_t* table = P.block_table + (long long)s * P.max_pages;
-    // Row numbers of this thread's rows of a tile of the selected list (-1 past the end).  They are fetched one
-    // tile ahead and only looked at when that tile's copies are issued, so the loader never waits on them.
+    // Row numbers of this warp's rows of a tile of the selected list (-1 past the end), `base` = the tile's first
+    // list entry, `count` = entries left from there.  The warp's RPT * ROWS_PER_INSTR rows are numbered
+    // p = i * ROWS_PER_INSTR + rsub; lane l keeps rows p = l and p = 32 + l (two registers instead of one per row
+    // group), and the thread that copies row p fetches its number with a shuffle.  Except for the first list tile
+    // they are fetched when the previous tile's copies have been issued and only looked at when this tile's copies
+    // are issued (the loader normally waits for a free slot in between), so the loader does not wait on them.
     // The per-row code below is kept free of branches (clamped loads, selects): a branch per row costs a single
     // warp far more than the arithmetic it skips.
-    auto list_rows = [&](int j, int (&t)[RPT]) {
-      if (SPARSE && j < g.n_sel) {
-        const int last = g.cnt - 1 - j * kKeyTile;                 // last valid row of this tile (>= 0)
+    constexpr int LIST_REGS = (RPT * ROWS_PER_INSTR + 31) / 32;
+    static_assert(32 % ROWS_PER_INSTR == 0, "a row group's entries must sit in one register");
+    int t_list[LIST_REGS];
+    auto list_rows = [&](int base, int count) {
+      const int last = min(count, kKeyTile) - 1;                   // last valid row of the tile
+      if (last >= 0) {
 #pragma unroll
-        for (int i = 0; i < RPT; ++i) {
-          const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
-          const int v = __ldg(idx + j * kKeyTile + min(rr, last));
-          t[i] = rr <= last ? v : -1;
+        for (int k = 0; k < LIST_REGS; ++k) {
+          const int pp = 32 * k + lane;
+          const int rr = (lw + (pp / ROWS_PER_INSTR) * kLoaderWarps) * ROWS_PER_INSTR + pp % ROWS_PER_INSTR;
+          const int v = __ldcg(idx + base + min(rr, last));        // written by the kernel before: L2, not the read-only path
+          t_list[k] = rr <= last ? v : -1;
         }
       }
     };
-    int t_cur[RPT], t_next[RPT];
 #pragma unroll
-    for (int i = 0; i < RPT; ++i) t_next[i] = -1;
-    list_rows(0, t_next);
-    for (int it = 0; it < n_items; ++it) {
-      if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) break;
-      const int j = it >> 1;
-      const bool from_list = SPARSE && j < g.n_sel;
-      if (!(it & 1)) {
-#pragma unroll
-        for (int i = 0; i < RPT; ++i) t_cur[i] = t_next[i];
+    for (int k = 0; k < LIST_REGS; ++k) t_list[k] = -1;
+    for (int tile = 0;; ++tile) {
+      if (tile == g.n_known) {                                // end of what is known: the list length, or the end
+        if (g.resolved) break;
+        resolve(g, k_cnt, s);
+        if (tile == g.n_known) break;
       }
-      // rows outside the list are consecutive: row_first + r for r < row_count (the chunk's own rows, or all rows)
-      int row_first, row_count;
-      if (SPARSE) { row_first = g.T + (j - g.n_sel) * kKeyTile; row_count = P.chunk - (j - g.n_sel) * kKeyTile; }
-      else { row_first = j * kKeyTile; row_count = g.T + P.chunk - j * kKeyTile; }
-      const uint4* src_base = reinterpret_cast<const uint4*>((it & 1) ? vc : kc);
-      const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
-      int t[RPT];                                                 // row number, or -1
-#pragma unroll
-      for (int i = 0; i < RPT; ++i) {
-        const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
-        t[i] = from_list ? t_cur[i] : (rr < row_count ? row_first + rr : -1);
-      }
-      uint32_t off[RPT];
-      if (P.page_size == 0) {
-#pragma unroll
-        for (int i = 0; i < RPT; ++i) off[i] = base16 + (uint32_t)max(t[i], 0) * st16;
-      } else {
+      const TileRows tr = tile_rows<SPARSE>(g, tile);
+      bool stop = false;
+#pragma unroll 1
+      for (int kvi = 0; kvi < 2; ++kvi) {                     // the tile's K rows, then its V rows
+        if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) { stop = true; break; }
+        if (kvi == 0 && tr.from_list && tile == g.n_chunk) list_rows(tr.first, tr.count);   // first list tile
+        const uint4* src_base = reinterpret_cast<const uint4*>(kvi ? vc : kc);
+        const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
+        int t[RPT];                                               // row number, or -1
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
-          const int tc = max(t[i], 0);
-          off[i] = (uint32_t)__ldg(table + (tc >> 6)) * sb16 + base16 + (uint32_t)(tc & (kPage - 1)) * st16;
+          const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
+          const int listed = __shfl_sync(0xFFFFFFFFu, t_list[(i * ROWS_PER_INSTR) / 32], (i * ROWS_PER_INSTR + rsub) & 31);
+          t[i] = tr.from_list ? listed : (rr < tr.count ? tr.first + rr : -1);
         }
-      }
+        uint32_t off[RPT];
+        if (P.page_size == 0) {
 #pragma unroll
-      for (int i = 0; i < RPT; ++i) {
-        const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
-        if (rr < kKeyTile)                                        // false only for the last group of some warps
-          cp_async_16(dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4), src_base + off[i], t[i] >= 0);
+          for (int i = 0; i < RPT; ++i) off[i] = base16 + (uint32_t)max(t[i], 0) * st16;
+        } else {
+#pragma unroll
+          for (int i = 0; i < RPT; ++i) {
+            const int tc = max(t[i], 0);
+            off[i] = (uint32_t)__ldg(table + (tc >> 6)) * sb16 + base16 + (uint32_t)(tc & (kPage - 1)) * st16;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) {
+          const int rr = (lw + i * kLoaderWarps) * ROWS_PER_INSTR + rsub;
+          if (rr < kKeyTile)                                      // false only for the last group of some warps
+            cp_async_16(dst_tile + rr * 128 + (((c16 & 7) ^ (rr & 7)) << 4), src_base + off[i], t[i] >= 0);
+        }
+        // this thread's share of the slot is signalled by the copy engine itself when the bytes have landed:
+        // no wait in the loader, every slot of the ring can be in flight
+        cp_async_mbar_arrive_noinc(&kv_full[slot]);
+        if (kvi == 1 && tr.from_list) list_rows(tr.first + kKeyTile, tr.count - kKeyTile);   // next list tile
+        if (++slot == kSlots) { slot = 0; phase ^= 1; }
       }
-      // this thread's share of the slot is signalled by the copy engine itself when the bytes have landed:
-      // no wait in the loader, every slot of the ring can be in flight
-      cp_async_mbar_arrive_noinc(&kv_full[slot]);
-      if (!(it & 1)) list_rows(j + 1, t_next);
-      if (++slot == kSlots) { slot = 0; phase ^= 1; }
+      if (stop) break;
     }
     cp_async_wait_all();                                      // nothing of this thread is in flight at exit
   } else if (lane == 0) {
@@ -389,7 +462,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
         }
       mma_commit(&s_full[x]);
     };
-    auto issue_pv = [&](int x, int vs, int j) {
+    auto issue_pv = [&](int x, int vs, bool first) {
       const uint64_t dv = desc_v + (uint64_t)((uint32_t)vs * (kTileBytes >> 4));
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
@@ -398,39 +471,43 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 #pragma unroll
         for (int kk = half * 4; kk < half * 4 + 4; ++kk) {   // 16 keys per MMA: 8 packed columns of P, 16 rows of V
           mma_ts(tmem_base + O_COL[x], tmem_base + S_COL[x] + kk * 8, dv + (uint64_t)(kk * (2048 >> 4)), idesc_pv,
-                 (j | kk) ? 1u : 0u);
+                 (!first || kk) ? 1u : 0u);
         }
       }
       p_phase[x] ^= 1;
     };
-    if (ok && g.n_max > 0) {
+    // Tile t: O += P_t V_t for each Q tile taking part (as the two halves of P arrive), then S = Q K_{t+1}^T.
+    // K_{t+1} and V_t are both acquired before the P waits, so those never sit on the P -> PV -> QK chain.
+    // The sparse sequence's length is learnt (resolve) just before the look-ahead past the chunk's own tiles.
+    const auto part = [&](int x, int t) { return x ? g.active_b : t >= g.skip_a; };
+    if (ok) {
       k_slot = acquire();
       if (ok) {
-        if (g.n_a > 0) issue_qk(0, k_slot);
-        if (g.n_b > 0) issue_qk(1, k_slot);
+        if (part(0, 0)) issue_qk(0, k_slot);
+        if (part(1, 0)) issue_qk(1, k_slot);
         mma_commit(&kv_empty[k_slot]);
       }
-      for (int j = 0; ok && j < g.n_max; ++j) {
-        const bool more = j + 1 < g.n_max;
+      for (int t = 0; ok; ++t) {
+        if (t + 1 == g.n_known && !g.resolved) resolve(g, k_cnt, s);
+        const bool more = t + 1 < g.n_known;
         v_slot = acquire();
-        if (ok && more) k_slot = acquire();     // both are normally there already: keeps the waits off the P -> PV -> QK chain
+        if (ok && more) k_slot = acquire();
         if (!ok) break;
-        if (j < g.n_a) {
-          issue_pv(0, v_slot, j);
+        if (part(0, t)) {
+          issue_pv(0, v_slot, t == g.skip_a);
           if (!ok) break;
-          if (j + 1 == g.n_a) mma_commit(&o_full[0]);
+          if (!more) mma_commit(&o_full[0]);
         }
-        if (more && j + 1 < g.n_a) issue_qk(0, k_slot);
-        if (j < g.n_b) {
-          issue_pv(1, v_slot, j);
+        if (more && part(0, t + 1)) issue_qk(0, k_slot);
+        if (part(1, t)) {
+          issue_pv(1, v_slot, t == 0);
           if (!ok) break;
-          if (j + 1 == g.n_b) mma_commit(&o_full[1]);
+          if (!more) mma_commit(&o_full[1]);
         }
         mma_commit(&kv_empty[v_slot]);
-        if (more) {
-          if (j + 1 < g.n_b) issue_qk(1, k_slot);
-          mma_commit(&kv_empty[k_slot]);
-        }
+        if (!more) break;
+        if (part(1, t + 1)) issue_qk(1, k_slot);
+        mma_commit(&kv_empty[k_slot]);
       }
     }
   }
@@ -449,7 +526,8 @@ bool attn_tc_supported(const quoka_params* p) {
 }
 
 quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
-                            const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st) {
+                            const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
+                            bool after_selection) {
   CUtensorMap tm_q;
   {
     const uint64_t dims[4] = {(uint64_t)P.d, (uint64_t)P.chunk, (uint64_t)P.n_q, (uint64_t)P.batch};
@@ -463,13 +541,28 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
   dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.batch);
   const bool sparse = k_idx != nullptr;
   cudaError_t e = cudaSuccess;
+  // Inside the fused call the sparse kernel is launched with programmatic stream serialisation: it may start
+  // while the kernel before it on the stream (the key selection, which signals early and writes none of this
+  // kernel's other inputs) still runs; it touches the selection's outputs only after its own
+  // griddepcontrol.wait.  A stand-alone call keeps the ordinary stream order: whatever ran before it may have
+  // written q, k or v.
 #define QUOKA_ATTN_TC(H, S)                                                                                      \
   do {                                                                                                           \
     e = cudaFuncSetAttribute(attn_tc_kernel<H, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                 \
-    attn_tc_kernel<H, S><<<grid, kAttnThreads, smem, st>>>(P, tm_q, (const __nv_bfloat16*)k,                     \
-                                                           (const __nv_bfloat16*)v, k_idx, k_cnt,                \
-                                                           (__nv_bfloat16*)out, lse);                            \
+    cudaLaunchConfig_t cfg = {};                                                                                 \
+    cfg.gridDim = grid;                                                                                          \
+    cfg.blockDim = dim3(kAttnThreads);                                                                           \
+    cfg.dynamicSmemBytes = smem;                                                                                 \
+    cfg.stream = st;                                                                                             \
+    cudaLaunchAttribute attr[1];                                                                                 \
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                             \
+    attr[0].val.programmaticStreamSerializationAllowed = 1;                                                      \
+    cfg.attrs = attr;                                                                                            \
+    cfg.numAttrs = ((S) && after_selection) ? 1 : 0;                                                                                \
+    e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<H, S>, P, tm_q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, \
+                           k_idx, k_cnt, (__nv_bfloat16*)out, lse);                                              \
+    if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                 \
   } while (0)
   if (halves == 2) { if (sparse) QUOKA_ATTN_TC(2, true); else QUOKA_ATTN_TC(2, false); }
   else { if (sparse) QUOKA_ATTN_TC(1, true); else QUOKA_ATTN_TC(1, false); }

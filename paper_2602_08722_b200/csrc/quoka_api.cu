@@ -138,8 +138,10 @@ static quoka_status run_score_keys(const quoka_params* p, const DevParams& P, co
 }
 
 static quoka_status run_attn(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
-                             const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st) {
-  if (use_tensor(p) && attn_tc_supported(p)) return launch_attn_tc(p, P, q, k, v, k_idx, k_cnt, out, lse, st);
+                             const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
+                             bool after_selection = false) {
+  if (use_tensor(p) && attn_tc_supported(p))
+    return launch_attn_tc(p, P, q, k, v, k_idx, k_cnt, out, lse, st, after_selection);
   if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;
   QUOKA_TRY_CUDA(launch_attn_simt(P, p->dtype, q, k, v, k_idx, k_cnt, out, lse, st));
   return QUOKA_OK;
@@ -247,7 +249,7 @@ quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const voi
   }
   // with an empty cache the selection kernel only writes k_cnt = 0 and the -1 padding
   QUOKA_TRY_CUDA(launch_select_keys(P, w.scores, k_idx, k_cnt, cs));
-  return run_attn(p, P, q, k_cache, v_cache, k_idx, k_cnt, out, nullptr, cs);
+  return run_attn(p, P, q, k_cache, v_cache, k_idx, k_cnt, out, nullptr, cs, /*after_selection=*/true);
 }
 
 quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_len_host, const void* q_host,

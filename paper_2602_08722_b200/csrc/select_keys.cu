@@ -33,6 +33,8 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_kernel(DevParams P, c
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t warp_off[33];
 
+  // the attention kernel that follows may start now: it waits for this grid itself before it reads the list
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int s = blockIdx.x / P.n_kv, kv = blockIdx.x % P.n_kv;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int T = __ldg(P.ctx_len + s);
@@ -141,6 +143,8 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   __shared__ uint32_t warp_off[33];
   __shared__ uint32_t cta_cnt[2];               // rows of this CTA above / equal to the threshold
 
+  // the attention kernel that follows may start now: it waits for this grid itself before it reads the list
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
   const int head = blockIdx.x / CL;

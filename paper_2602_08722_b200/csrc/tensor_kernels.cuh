@@ -12,6 +12,7 @@ quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, con
 
 bool attn_tc_supported(const quoka_params* p);
 quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
-                            const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st);
+                            const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
+                            bool after_selection);
 
 }  // namespace quoka
