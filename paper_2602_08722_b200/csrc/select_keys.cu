@@ -165,14 +165,41 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   }
   const int base = (rank * kSelThreads + wid * 32) * ITEMS + lane;      // position of item i: base + 32 i
   uint32_t code[ITEMS];
+  uint32_t cmin = 0xFFFFFFFFu, cmax = 0u;
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
     const int pos = base + 32 * i;
     const uint32_t c = float_order_key(__ldg(row + min(pos, T - 1)));      // clamped load, no branch per item
-    code[i] = pos < T ? c : 0u;
+    code[i] = c;                                                           // (a row past the end repeats the last one)
+    cmin = min(cmin, c);
+    cmax = max(cmax, c);
   }
   for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
+  // The codes of one row of scores share their leading bits (cosines of similar size): digits of the raw code
+  // would put most rows into a few bins, which serialises the shared-memory atomics and leaves every pass
+  // with many rows.  The digits are taken from (code - smallest code) shifted up to the top bit instead; the map
+  // keeps the order, and no bit is lost.
+  cmin = __reduce_min_sync(0xFFFFFFFFu, cmin);
+  cmax = __reduce_max_sync(0xFFFFFFFFu, cmax);
+  if (lane == 0) { warp_val[wid] = cmin; warp_off[wid] = cmax; }
   __syncthreads();
+  cmin = __reduce_min_sync(0xFFFFFFFFu, warp_val[lane]);
+  cmax = __reduce_max_sync(0xFFFFFFFFu, warp_off[lane]);
+  if (CL > 1) {
+    if (tid == 0) { cta_cnt[0] = cmin; cta_cnt[1] = cmax; }
+    cluster.sync();
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+      const uint32_t* pc = cluster.map_shared_rank(cta_cnt, r);
+      cmin = min(cmin, pc[0]);
+      cmax = max(cmax, pc[1]);
+    }
+    cluster.sync();                                // cta_cnt is used again below
+  }
+  const int up = min(__clz((int)(cmax - cmin)), 31);
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) code[i] = (code[i] - cmin) << up;
+  __syncthreads();                                 // the histograms are zero, warp_val / warp_off free again
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t prefix = 0, mask = 0, need = (uint32_t)B;
 #pragma unroll 1
@@ -241,66 +268,100 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     need = s_need;
     mask |= (uint32_t)(nb - 1) << shift;
   }
-  // prefix = code of the B-th largest score; take every row above it and the first `need` rows equal to it
+  // prefix = (shifted) code of the B-th largest score.  Rows at or above it, per warp and before each warp:
   const uint32_t thr = prefix;
-  uint32_t w_gt = 0, w_eq = 0;
+  uint32_t w_ge = 0;
 #pragma unroll
-  for (int i = 0; i < ITEMS; ++i) {
-    const bool in = base + 32 * i < T;
-    w_gt += (in && code[i] > thr) ? 1u : 0u;
-    w_eq += (in && code[i] == thr) ? 1u : 0u;
-  }
-  w_gt = __reduce_add_sync(0xFFFFFFFFu, w_gt);
-  w_eq = __reduce_add_sync(0xFFFFFFFFu, w_eq);
-  if (lane == 0) warp_val[wid] = w_gt | (w_eq << 16);      // at most 1024 each
+  for (int i = 0; i < ITEMS; ++i) w_ge += (base + 32 * i < T && code[i] >= thr) ? 1u : 0u;
+  w_ge = __reduce_add_sync(0xFFFFFFFFu, w_ge);
+  if (lane == 0) warp_val[wid] = w_ge;
   __syncthreads();
   if (wid == 0) {
     const uint32_t v = warp_val[lane];
-    uint32_t g = v & 0xFFFFu, e = v >> 16, gi = g, ei = e;
+    uint32_t vi = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t ug = __shfl_up_sync(0xFFFFFFFFu, gi, o), ue = __shfl_up_sync(0xFFFFFFFFu, ei, o);
-      if (lane >= o) { gi += ug; ei += ue; }
+      const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, vi, o);
+      if (lane >= o) vi += u;
     }
-    warp_off[lane] = gi - g;                 // exclusive counts of rows above the threshold ...
-    warp_val[lane] = ei - e;                 // ... and equal to it, over the warps before this one
-    if (lane == 31) { cta_cnt[0] = gi; cta_cnt[1] = ei; }
+    warp_off[lane] = vi - v;                 // rows at or above the threshold in the warps before this one
+    if (lane == 31) cta_cnt[0] = vi;
   }
   if (CL > 1) cluster.sync(); else __syncthreads();
-  uint32_t run_gt = warp_off[wid], run_eq = warp_val[wid];
-  uint32_t total_eq = cta_cnt[1];
+  uint32_t run = warp_off[wid];
+  uint32_t total_ge = cta_cnt[0];
   if (CL > 1) {
-    uint32_t pg[CL], pe[CL];
+    uint32_t pg[CL];
 #pragma unroll
-    for (int r = 0; r < CL; ++r) {               // independent remote loads
-      const uint32_t* pc = cluster.map_shared_rank(cta_cnt, r);
-      pg[r] = pc[0];
-      pe[r] = pc[1];
-    }
-    total_eq = 0;
+    for (int r = 0; r < CL; ++r) pg[r] = cluster.map_shared_rank(cta_cnt, r)[0];      // independent remote loads
+    total_ge = 0;
 #pragma unroll
     for (int r = 0; r < CL; ++r) {
-      total_eq += pe[r];
-      if (r < rank) { run_gt += pg[r]; run_eq += pe[r]; }
+      total_ge += pg[r];
+      if (r < rank) run += pg[r];
     }
   }
-  if (need == total_eq) {
-    // every row equal to the threshold is taken (no tie is cut): one predicate, one ballot per item
-    uint32_t run = run_gt + run_eq;
+  if (total_ge == (uint32_t)B) {
+    // No tie is cut (the usual case): the list is every row at or above the threshold, one ballot per item.
+    // A single CTA collects the list in shared memory (over the histograms, which are done with) and copies
+    // it out with full-width stores; a cluster writes straight to the list.
+    const bool staged = CL == 1 && B <= kHistWords;
+    uint32_t* dst = staged ? hist_all : reinterpret_cast<uint32_t*>(out);
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       const int pos = base + 32 * i;
       const bool sel = pos < T && code[i] >= thr;
-      const uint32_t b = __ballot_sync(0xFFFFFFFFu, sel);
-      if (sel) out[run + (uint32_t)__popc(b & lt)] = pos;
-      run += (uint32_t)__popc(b);
+      const uint32_t bal = __ballot_sync(0xFFFFFFFFu, sel);
+      if (sel) dst[run + (uint32_t)__popc(bal & lt)] = (uint32_t)pos;
+      run += (uint32_t)__popc(bal);
+    }
+    if (staged) {
+      __syncthreads();
+      for (int i = tid; i < B; i += kSelThreads) out[i] = (int32_t)hist_all[i];
     }
   } else {
-#pragma unroll
+    // Rows that tie at the threshold and do not all fit: take the first `need` of them in position order.
+    // Rare, so the codes are rebuilt from the scores one item at a time instead of keeping a second unrolled
+    // loop over the registers (which made the compiler spill fifty of them).
+    uint32_t w_gt = 0, w_eq = 0;
+#pragma unroll 1
     for (int i = 0; i < ITEMS; ++i) {
       const int pos = base + 32 * i;
-      const bool in = pos < T;
-      const bool gt = in && code[i] > thr, eq = in && code[i] == thr;
+      const uint32_t c = (float_order_key(__ldg(row + min(pos, T - 1))) - cmin) << up;
+      w_gt += (pos < T && c > thr) ? 1u : 0u;
+      w_eq += (pos < T && c == thr) ? 1u : 0u;
+    }
+    w_gt = __reduce_add_sync(0xFFFFFFFFu, w_gt);
+    w_eq = __reduce_add_sync(0xFFFFFFFFu, w_eq);
+    if (CL > 1) cluster.sync(); else __syncthreads();        // warp_val / warp_off / cta_cnt were read above
+    if (lane == 0) warp_val[wid] = w_gt | (w_eq << 16);      // at most 1024 each
+    __syncthreads();
+    if (wid == 0) {
+      const uint32_t v = warp_val[lane];
+      uint32_t g = v & 0xFFFFu, e = v >> 16, gi = g, ei = e;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t ug = __shfl_up_sync(0xFFFFFFFFu, gi, o), ue = __shfl_up_sync(0xFFFFFFFFu, ei, o);
+        if (lane >= o) { gi += ug; ei += ue; }
+      }
+      warp_off[lane] = gi - g;                 // exclusive counts of rows above the threshold ...
+      warp_val[lane] = ei - e;                 // ... and equal to it, over the warps before this one
+      if (lane == 31) { cta_cnt[0] = gi; cta_cnt[1] = ei; }
+    }
+    if (CL > 1) cluster.sync(); else __syncthreads();
+    uint32_t run_gt = warp_off[wid], run_eq = warp_val[wid];
+    if (CL > 1) {
+#pragma unroll
+      for (int r = 0; r < CL; ++r) {
+        const uint32_t* pc = cluster.map_shared_rank(cta_cnt, r);
+        if (r < rank) { run_gt += pc[0]; run_eq += pc[1]; }
+      }
+    }
+#pragma unroll 1
+    for (int i = 0; i < ITEMS; ++i) {
+      const int pos = base + 32 * i;
+      const uint32_t c = (float_order_key(__ldg(row + min(pos, T - 1))) - cmin) << up;
+      const bool gt = pos < T && c > thr, eq = pos < T && c == thr;
       const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt), b_eq = __ballot_sync(0xFFFFFFFFu, eq);
       const uint32_t gt_before = run_gt + (uint32_t)__popc(b_gt & lt);
       const uint32_t eq_before = run_eq + (uint32_t)__popc(b_eq & lt);
