@@ -132,20 +132,60 @@ __device__ __forceinline__ float warp_sum(float x) {
   return x;
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------
+// The kernels of one fused call form a chain on one stream, each reading what the one before it wrote.  A kernel
+// launched with programmatic stream serialisation may become resident while the kernel before it still runs;
+// it must then execute grid_dependency_wait() before its first access to anything that kernel writes (the wait
+// returns once that grid has completed and its writes are visible; without the launch attribute it returns at
+// once).  A kernel lets the one after it start early with grid_launch_dependents(), which every CTA executes at
+// its start; the dependent grid is launched when all of them have, so it never holds resources that this
+// grid's own CTAs still need.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Launch with optional thread-block cluster width and, if `chained`, programmatic stream serialisation.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 int cluster, bool chained, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (chained) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- launch functions implemented in the .cu files (host side) -------------------------------
+// `chained`: the kernel before it on the stream is the one of the same fused call whose output it reads (see above).
 struct Launch {
   cudaStream_t stream;
 };
 
 cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st);
 cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, const int32_t* q_idx, void* qbar,
-                                     cudaStream_t st);
+                                     cudaStream_t st, bool chained = false);
 cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,
                                    cudaStream_t st);
 cudaError_t launch_key_norms(const DevParams& P, int dtype, const void* k, float* k_inv_norm, int all_rows,
                              cudaStream_t st);
 cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt,
-                               cudaStream_t st);
+                               cudaStream_t st, bool chained = false);
 cudaError_t launch_attn_simt(const DevParams& P, int dtype, const void* q, const void* k, const void* v,
                              const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st);
 

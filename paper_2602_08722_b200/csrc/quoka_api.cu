@@ -124,14 +124,15 @@ static bool use_tensor(const quoka_params* p) {
 static quoka_status run_select_queries(const quoka_params* p, const DevParams& P, const void* q, int32_t* q_idx,
                                        void* qbar, cudaStream_t st) {
   QUOKA_TRY_CUDA(launch_rank_queries(P, p->dtype, q, q_idx, st));
-  QUOKA_TRY_CUDA(launch_aggregate_queries(P, p->dtype, q, q_idx, qbar, st));
+  QUOKA_TRY_CUDA(launch_aggregate_queries(P, p->dtype, q, q_idx, qbar, st, /*chained=*/true));
   return QUOKA_OK;
 }
 
+// chained: the aggregation kernel of the same call is the kernel before it on the stream
 static quoka_status run_score_keys(const quoka_params* p, const DevParams& P, const void* qbar, const void* k,
-                                   float* scores, cudaStream_t st) {
+                                   float* scores, cudaStream_t st, bool chained = false) {
   if (p->max_ctx_len == 0) return QUOKA_OK;
-  if (use_tensor(p) && score_keys_tc_supported(p)) return launch_score_keys_tc(p, P, qbar, k, scores, st);
+  if (use_tensor(p) && score_keys_tc_supported(p)) return launch_score_keys_tc(p, P, qbar, k, scores, st, chained);
   if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;
   QUOKA_TRY_CUDA(launch_score_keys_simt(P, p->dtype, qbar, k, scores, st));
   return QUOKA_OK;
@@ -245,10 +246,10 @@ quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const voi
   int32_t* k_cnt = k_cnt_out ? k_cnt_out : w.k_cnt;
   if (p->max_ctx_len > 0) {
     if ((st = run_select_queries(p, P, q, w.q_idx, w.qbar, cs)) != QUOKA_OK) return st;
-    if ((st = run_score_keys(p, P, w.qbar, k_cache, w.scores, cs)) != QUOKA_OK) return st;
+    if ((st = run_score_keys(p, P, w.qbar, k_cache, w.scores, cs, /*chained=*/true)) != QUOKA_OK) return st;
   }
   // with an empty cache the selection kernel only writes k_cnt = 0 and the -1 padding
-  QUOKA_TRY_CUDA(launch_select_keys(P, w.scores, k_idx, k_cnt, cs));
+  QUOKA_TRY_CUDA(launch_select_keys(P, w.scores, k_idx, k_cnt, cs, /*chained=*/p->max_ctx_len > 0));
   return run_attn(p, P, q, k_cache, v_cache, k_idx, k_cnt, out, nullptr, cs, /*after_selection=*/true);
 }
 

@@ -54,6 +54,7 @@ static ScoreSmemPlan plan_score_smem(int N, int d) {
 
 struct ScoreArgs {
   int n, n_pad, n_parts, box_rows, q_rows, stages;
+  int defer_q;   // launched early (chained): fetch the key tiles that fit the ring before the first Q-bar
 };
 
 // Walks the valid (sequence, KV head, tile) triples in linear order.
@@ -114,6 +115,7 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{&abort_flag, P.status};
+  grid_launch_dependents();                  // the selection kernel may become resident; it waits for this grid itself
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -140,15 +142,25 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
     if (lane == 0) {
       TileWalk w; w.seek(P, lo, hi);
       int stage = 0; uint32_t phase = 0, qe_phase = 0; int head_cur = -1;
+      // The key tiles do not depend on the kernel before this one, Q-bar does.  The first Q-bar of the CTA is
+      // therefore fetched only after most of the ring has been filled with key tiles, and after the wait for the
+      // grid that wrote it (which returns at once unless this kernel was launched early).
+      bool waited = false;
+      int q_deferred = -1, n_issued = 0;
+      const auto load_q = [&](int head) {
+        if (!waited) { grid_dependency_wait(); waited = true; }
+        mbar_arrive_expect_tx(q_full, (uint32_t)(HALVES * A.n_parts * A.box_rows * 128));
+        for (int h = 0; h < HALVES; ++h)
+          for (int p = 0; p < A.n_parts; ++p)
+            tma_load_3d(q_smem + (size_t)h * q_half_bytes + (size_t)p * A.box_rows * 128, &tm_q, q_full, h * 64,
+                        p * A.box_rows, head);
+      };
       for (; w.valid(); w.next(P)) {
         const int head = w.s * P.n_kv + w.kv;
         if (head != head_cur) {
+          if (q_deferred >= 0) { load_q(q_deferred); q_deferred = -1; }
           if (head_cur >= 0) { if (!mbar_wait(q_empty, qe_phase, wc)) break; qe_phase ^= 1; }
-          mbar_arrive_expect_tx(q_full, (uint32_t)(HALVES * A.n_parts * A.box_rows * 128));
-          for (int h = 0; h < HALVES; ++h)
-            for (int p = 0; p < A.n_parts; ++p)
-              tma_load_3d(q_smem + (size_t)h * q_half_bytes + (size_t)p * A.box_rows * 128, &tm_q, q_full, h * 64,
-                          p * A.box_rows, head);
+          if (n_issued == 0 && A.defer_q) q_deferred = head; else load_q(head);
           head_cur = head;
         }
         if (!mbar_wait(&empty[stage], phase ^ 1, wc)) break;
@@ -169,7 +181,9 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
             tma_load_4d(dst + h * kHalfBytes + sub * 64 * 128, &tm_k, &full[stage], h * 64, c1, w.kv, c3);
         }
         if (++stage == A.stages) { stage = 0; phase ^= 1; }
+        if (++n_issued >= A.stages - 1 && q_deferred >= 0) { load_q(q_deferred); q_deferred = -1; }
       }
+      if (q_deferred >= 0) load_q(q_deferred);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -388,7 +402,7 @@ bool score_keys_tc_supported(const quoka_params* p) {
 }
 
 quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, const void* qbar, const void* k,
-                                  float* scores, cudaStream_t st) {
+                                  float* scores, cudaStream_t st, bool chained) {
   const int N = P.n_sel;
   const ScoreSmemPlan pl = plan_score_smem(N, P.d);
   if (pl.stages < 2) return QUOKA_ERR_UNSUPPORTED;
@@ -400,7 +414,7 @@ quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, con
     if (!encode_tensor_map_bf16(&tm_q, qbar, 3, dims, strides, box)) return QUOKA_ERR_CUDA;
   }
   if (!encode_kv_tensor_map(&tm_k, p, k, 64)) return QUOKA_ERR_CUDA;
-  ScoreArgs A{N, pl.n_pad, pl.n_parts, pl.box_rows, pl.q_rows, pl.stages};
+  ScoreArgs A{N, pl.n_pad, pl.n_parts, pl.box_rows, pl.q_rows, pl.stages, chained ? 1 : 0};
   const long long max_tiles = (long long)P.batch * P.n_kv * ((P.max_ctx + kTileKeys - 1) / kTileKeys);
   int grid = sm_count();
   if (grid <= 0) return QUOKA_ERR_CUDA;
@@ -410,14 +424,14 @@ quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, con
   if (P.d == 128) {
     e = cudaFuncSetAttribute(score_keys_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.total);
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;
-    score_keys_tc_kernel<2><<<grid, kScoreThreads, pl.total, st>>>(P, A, tm_q, tm_k, scores);
+    e = launch_kernel(score_keys_tc_kernel<2>, dim3(grid), dim3(kScoreThreads), pl.total, st, 1, chained, P, A, tm_q, tm_k, scores);
   } else {
     e = cudaFuncSetAttribute(score_keys_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.total);
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;
-    score_keys_tc_kernel<1><<<grid, kScoreThreads, pl.total, st>>>(P, A, tm_q, tm_k, scores);
+    e = launch_kernel(score_keys_tc_kernel<1>, dim3(grid), dim3(kScoreThreads), pl.total, st, 1, chained, P, A, tm_q, tm_k, scores);
   }
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? QUOKA_OK : QUOKA_ERR_CUDA;
+  return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? QUOKA_OK : QUOKA_ERR_CUDA;
 }
 
 }  // namespace quoka

@@ -33,8 +33,8 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_kernel(DevParams P, c
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t warp_off[33];
 
-  // the attention kernel that follows may start now: it waits for this grid itself before it reads the list
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  grid_launch_dependents();     // the attention kernel may start now: it waits for this grid itself before it reads the list
+  grid_dependency_wait();       // the scores come from the kernel before
   const int s = blockIdx.x / P.n_kv, kv = blockIdx.x % P.n_kv;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int T = __ldg(P.ctx_len + s);
@@ -143,8 +143,8 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   __shared__ uint32_t warp_off[33];
   __shared__ uint32_t cta_cnt[2];               // rows of this CTA above / equal to the threshold
 
-  // the attention kernel that follows may start now: it waits for this grid itself before it reads the list
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  grid_launch_dependents();     // the attention kernel may start now: it waits for this grid itself before it reads the list
+  grid_dependency_wait();       // the scores come from the kernel before
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
   const int head = blockIdx.x / CL;
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
     const int pos = base + 32 * i;
-    const uint32_t c = float_order_key(__ldg(row + min(pos, T - 1)));      // clamped load, no branch per item
+    const uint32_t c = float_order_key(__ldcg(row + min(pos, T - 1)));      // clamped load, no branch per item
     code[i] = c;                                                           // (a row past the end repeats the last one)
     cmin = min(cmin, c);
     cmax = max(cmax, c);
@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll 1
     for (int i = 0; i < ITEMS; ++i) {
       const int pos = base + 32 * i;
-      const uint32_t c = (float_order_key(__ldg(row + min(pos, T - 1))) - cmin) << up;
+      const uint32_t c = (float_order_key(__ldcg(row + min(pos, T - 1))) - cmin) << up;
       w_gt += (pos < T && c > thr) ? 1u : 0u;
       w_eq += (pos < T && c == thr) ? 1u : 0u;
     }
@@ -360,7 +360,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll 1
     for (int i = 0; i < ITEMS; ++i) {
       const int pos = base + 32 * i;
-      const uint32_t c = (float_order_key(__ldg(row + min(pos, T - 1))) - cmin) << up;
+      const uint32_t c = (float_order_key(__ldcg(row + min(pos, T - 1))) - cmin) << up;
       const bool gt = pos < T && c > thr, eq = pos < T && c == thr;
       const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt), b_eq = __ballot_sync(0xFFFFFFFFu, eq);
       const uint32_t gt_before = run_gt + (uint32_t)__popc(b_gt & lt);
@@ -374,40 +374,26 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 }
 
 template <int ITEMS, int CL>
-static cudaError_t launch_reg(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt, cudaStream_t st) {
-  if (CL == 1) {
-    select_keys_reg_kernel<ITEMS, CL><<<P.batch * P.n_kv, kSelThreads, 0, st>>>(P, scores, k_idx, k_cnt);
-    return cudaSuccess;
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(P.batch * P.n_kv * CL);
-  cfg.blockDim = dim3(kSelThreads);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = CL;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, select_keys_reg_kernel<ITEMS, CL>, P, scores, k_idx, k_cnt);
+static cudaError_t launch_reg(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt, cudaStream_t st,
+                              bool chained) {
+  return launch_kernel(select_keys_reg_kernel<ITEMS, CL>, dim3(P.batch * P.n_kv * CL), dim3(kSelThreads), 0, st, CL, chained,
+                       P, scores, k_idx, k_cnt);
 }
 
 cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt,
-                               cudaStream_t st) {
+                               cudaStream_t st, bool chained) {
   // One CTA per head while the row fits its registers (32 per thread); clusters only for longer rows: merging
   // the histograms through distributed shared memory costs more than it saves on a short row.
   const int per_thread = (P.max_ctx + kSelThreads - 1) / kSelThreads;    // items per thread with one CTA per head
   cudaError_t e;
-  if (per_thread <= 4) e = launch_reg<4, 1>(P, scores, k_idx, k_cnt, st);
-  else if (per_thread <= 8) e = launch_reg<8, 1>(P, scores, k_idx, k_cnt, st);
-  else if (per_thread <= 16) e = launch_reg<16, 1>(P, scores, k_idx, k_cnt, st);
-  else if (per_thread <= 32) e = launch_reg<32, 1>(P, scores, k_idx, k_cnt, st);
-  else if (per_thread <= 64) e = launch_reg<32, 2>(P, scores, k_idx, k_cnt, st);
-  else if (per_thread <= 128) e = launch_reg<32, 4>(P, scores, k_idx, k_cnt, st);
-  else if (per_thread <= 256) e = launch_reg<32, 8>(P, scores, k_idx, k_cnt, st);
-  else { select_keys_kernel<<<P.batch * P.n_kv, kSelThreads, 0, st>>>(P, scores, k_idx, k_cnt); e = cudaSuccess; }
+  if (per_thread <= 4) e = launch_reg<4, 1>(P, scores, k_idx, k_cnt, st, chained);
+  else if (per_thread <= 8) e = launch_reg<8, 1>(P, scores, k_idx, k_cnt, st, chained);
+  else if (per_thread <= 16) e = launch_reg<16, 1>(P, scores, k_idx, k_cnt, st, chained);
+  else if (per_thread <= 32) e = launch_reg<32, 1>(P, scores, k_idx, k_cnt, st, chained);
+  else if (per_thread <= 64) e = launch_reg<32, 2>(P, scores, k_idx, k_cnt, st, chained);
+  else if (per_thread <= 128) e = launch_reg<32, 4>(P, scores, k_idx, k_cnt, st, chained);
+  else if (per_thread <= 256) e = launch_reg<32, 8>(P, scores, k_idx, k_cnt, st, chained);
+  else e = launch_kernel(select_keys_kernel, dim3(P.batch * P.n_kv), dim3(kSelThreads), 0, st, 1, chained, P, scores, k_idx, k_cnt);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -51,6 +51,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams P, const T* __restrict__ q,
                                                                      int32_t* __restrict__ q_idx, int rpc, int n_sort,
                                                                      int staged, int m_peer) {
+  grid_launch_dependents();                 // the aggregation kernel may become resident; it waits for this grid itself
   constexpr int LG = D / 8;                 // lanes per row, 8 elements each
   constexpr int RPI = kRankThreads / LG;    // rows per iteration
   constexpr int NW = sizeof(T) * 8 / 16;    // 16-byte words per lane
@@ -307,6 +308,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, const T* __restrict__ q,
                                                                  const int32_t* __restrict__ q_idx,
                                                                  T* __restrict__ qbar) {
+  grid_launch_dependents();
+  grid_dependency_wait();                   // the ranks come from the kernel before
   constexpr int NE = D / 32;
   const int N = P.n_sel;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -322,7 +325,7 @@ __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, con
   for (int g0 = 0; g0 < P.group; g0 += 32) {
     // the group's ranks in one load, then the rows four at a time so their loads overlap
     const int gl = g0 + lane;
-    const int r_lane = gl < P.group ? __ldg(q_idx + ((int64_t)s * P.n_q + kv * P.group + gl) * N + j) : 0;
+    const int r_lane = gl < P.group ? __ldcg(q_idx + ((int64_t)s * P.n_q + kv * P.group + gl) * N + j) : 0;
     const int g_end = min(32, P.group - g0);
     for (int g4 = 0; g4 < g_end; g4 += 4) {
       float x[4][NE];
@@ -372,19 +375,8 @@ static cudaError_t launch_rank_t(const DevParams& P, const void* q, int32_t* q_i
   const size_t smem = fixed + (staged ? row_bytes : 0);
   cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(P.batch * P.n_q * kRankCluster);
-  cfg.blockDim = dim3(kRankThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kRankCluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, rank_queries_kernel<T, D>, P, (const T*)q, q_idx, rpc, n_sort, staged, m_peer);
+  return launch_kernel(rank_queries_kernel<T, D>, dim3(P.batch * P.n_q * kRankCluster), dim3(kRankThreads), smem, st, kRankCluster,
+                       false, P, (const T*)q, q_idx, rpc, n_sort, staged, m_peer);
 }
 
 cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st) {
@@ -396,16 +388,18 @@ cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, in
 }
 
 cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, const int32_t* q_idx, void* qbar,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, bool chained) {
   const int64_t warps = (int64_t)P.batch * P.n_kv * P.n_sel;
-  const int grid = (int)((warps * 32 + 255) / 256);
+  const dim3 grid((unsigned)((warps * 32 + 255) / 256)), block(256);
+  cudaError_t e;
   if (dtype == QUOKA_BF16) {
-    if (P.d == 128) aggregate_queries_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
-    else aggregate_queries_kernel<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
+    if (P.d == 128) e = launch_kernel(aggregate_queries_kernel<__nv_bfloat16, 128>, grid, block, 0, st, 1, chained, P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
+    else e = launch_kernel(aggregate_queries_kernel<__nv_bfloat16, 64>, grid, block, 0, st, 1, chained, P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
   } else {
-    if (P.d == 128) aggregate_queries_kernel<float, 128><<<grid, 256, 0, st>>>(P, (const float*)q, q_idx, (float*)qbar);
-    else aggregate_queries_kernel<float, 64><<<grid, 256, 0, st>>>(P, (const float*)q, q_idx, (float*)qbar);
+    if (P.d == 128) e = launch_kernel(aggregate_queries_kernel<float, 128>, grid, block, 0, st, 1, chained, P, (const float*)q, q_idx, (float*)qbar);
+    else e = launch_kernel(aggregate_queries_kernel<float, 64>, grid, block, 0, st, 1, chained, P, (const float*)q, q_idx, (float*)qbar);
   }
+  if (e != cudaSuccess) return e;
   count_launch();
   return cudaGetLastError();
 }

@@ -8,7 +8,7 @@ namespace quoka {
 // Whether the tensor-core kernel covers this configuration (bf16, supported N / head_dim / layout).
 bool score_keys_tc_supported(const quoka_params* p);
 quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, const void* qbar, const void* k,
-                                  float* scores, cudaStream_t st);
+                                  float* scores, cudaStream_t st, bool chained);
 
 bool attn_tc_supported(const quoka_params* p);
 quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
