@@ -255,6 +255,31 @@ def test_select_keys_exact_with_planted_ties(T, B):
     assert int(gp.k_cnt[0]) == B
 
 
+@pytest.mark.parametrize("T,B", [(4097, 500), (31000, 3720), (40000, 39999)])
+def test_select_keys_constant_and_narrow_rows(T, B):
+    """Rows whose codes span almost nothing (the digits are taken relative to the row's smallest code): a
+    constant row, a row of adjacent floats, a row with one outlier above a constant."""
+    s = np.empty((3, T), dtype=np.float32)
+    s[0, :] = 0.3125                                             # every score ties: the first B positions win
+    base = np.float32(0.4)
+    s[1, :] = base
+    steps = np.random.default_rng(T).integers(0, 6, T)           # 0..5 ulps above the base, many ties per value
+    for k in range(1, 6):
+        v = base
+        for _ in range(k):
+            v = np.nextafter(v, np.float32(1.0))
+        s[1, steps == k] = v
+    s[2, :] = -0.75
+    s[2, T // 2] = 0.9
+    inp = synth.make_chunk_inputs(0, 1, 3, 3, 64, T, 8, "bf16")
+    gp = GpuProblem(inp, 4, kv_budget=B)
+    gp.scores[0, :, :T] = torch.from_numpy(s).cuda()
+    api.quoka_select_keys(gp.p, gp.scores, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    want = O.select_keys(s.astype(np.float64), B)
+    np.testing.assert_array_equal(gp.k_idx[0, :, :B].cpu().numpy(), want)
+
+
 # ---------------------------------------------------------------- full-size configurations
 def test_llama8b_32k_full_size():
     w = synth.WORKLOADS["llama8b_32k"]
