@@ -7,7 +7,7 @@
 // the key tiles (128 keys) once for both.  Roles:
 //   warps 0-3 / 4-7  softmax of Q tile A / B: one thread per query row, S read from tensor memory,
 //                    running max / sum in registers, P written back to tensor memory over S,
-//                    lazy rescale of the O accumulator (only when the max grew by more than 2^8),
+//                    lazy rescale of the O accumulator (only when the max grew by more than 2^32),
 //                    final normalisation and the global store.
 //   warps 8-10       loaders: every K / V row of a tile is fetched with 16-byte cp.async straight
 //                    into the 128-byte-swizzled layout the MMA descriptors expect.  The row address
@@ -34,7 +34,12 @@ constexpr int kMmaWarp = 11;
 constexpr int kQTile = 128;
 constexpr int kKeyTile = 128;
 constexpr int kSlots = 5;
-constexpr float kRescaleThreshold = 8.0f;   // log2 units
+// The reference point m of the exponentials 2^(s - m) is raised, and O and l rescaled, only when a row's maximum
+// exceeds it by more than this many powers of two.  Until then P, l and O are simply larger by a common factor of at
+// most 2^32, which floating point carries without loss (bf16 and fp32 both reach 2^127; l <= 2^32 * keys and
+// |O| <= l * max|v| stay far below that); the quotient O / l does not change.  With 8 the rescale (a read-modify-
+// write of the whole accumulator row on the softmax -> PV chain) still ran often enough to cost 1-2 % of the kernel.
+constexpr float kRescaleThreshold = 32.0f;   // log2 units
 
 bool encode_kv_tensor_map(CUtensorMap* out, const quoka_params* p, const void* cache, uint32_t box_rows);
 
