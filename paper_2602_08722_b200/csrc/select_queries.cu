@@ -7,7 +7,7 @@
 //                through distributed shared memory in a fixed order.  Pass 2 computes
 //                CosSim(q_r, M) for every row of the slice from shared memory, sorts the slice's
 //                (cosine, position) codes with a shared-memory bitonic sort, and places each of its
-//                N smallest by global rank: own rank + binary searches in the seven peers' sorted
+//                N smallest by global rank: own rank + binary searches in the peers' sorted
 //                slices.  Codes are unique (the position is part of them), so the N lowest cosines
 //                come out in ascending order, equal cosines by position.
 // aggregate    : one warp per (sequence, KV head, rank j): mean over the G heads of the group of
@@ -47,7 +47,7 @@ __device__ __forceinline__ void raw_to_f32(const Raw8<T>& r, float (&x)[8]) {
   }
 }
 
-template <typename T, int D>
+template <typename T, int D, int CL>
 __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams P, const T* __restrict__ q,
                                                                      int32_t* __restrict__ q_idx, int rpc, int n_sort,
                                                                      int staged, int m_peer) {
@@ -62,21 +62,21 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
   float* red = reinterpret_cast<float*>(smem_raw + (size_t)n_sort * 16);                    // [RPI][D]
   float* norms = red + RPI * D;                                                             // [rpc]
   unsigned long long* peer_keys = reinterpret_cast<unsigned long long*>(norms + ((rpc + 3) & ~3));   // [7][m_peer]
-  uint4* rows = reinterpret_cast<uint4*>(peer_keys + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1));   // [rpc][LG][NW]
+  uint4* rows = reinterpret_cast<uint4*>(peer_keys + (((size_t)(CL - 1) * m_peer + 1) & ~(size_t)1));   // [rpc][LG][NW]
   __shared__ float part[D];                 // this CTA's share of the column sums
   __shared__ __align__(16) float M[D];
   __shared__ float Mnorm;
 
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
-  const int head = blockIdx.x / kRankCluster;
+  const int head = blockIdx.x / CL;
   const int s = head / P.n_q, h = head % P.n_q;
   const int C = P.chunk, N = P.n_sel;
   int32_t* out = q_idx + (long long)head * N;
   const int tid = threadIdx.x;
 
   if (C <= P.n_retain) {                    // no sub-selection: every query, in position order
-    for (int j = rank * kRankThreads + tid; j < C; j += kRankCluster * kRankThreads) out[j] = j;
+    for (int j = rank * kRankThreads + tid; j < C; j += CL * kRankThreads) out[j] = j;
     return;
   }
 
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
   if (tid < D) {
     float sum = 0.f;
 #pragma unroll
-    for (int r = 0; r < kRankCluster; ++r) sum += cluster.map_shared_rank(part, r)[tid];   // fixed order
+    for (int r = 0; r < CL; ++r) sum += cluster.map_shared_rank(part, r)[tid];   // fixed order
     M[tid] = sum / (float)C;
   }
   __syncthreads();
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
   // peer's first m_peer codes matter (m_peer = a power of two >= min(n_sort, N): more smaller ones than N
   // already push the rank past N); they are copied into local shared memory first, because a chain of
   // dependent remote reads is slow.
-  for (int e = tid; e < (kRankCluster - 1) * m_peer; e += kRankThreads) {
+  for (int e = tid; e < (CL - 1) * m_peer; e += kRankThreads) {
     const int pr = e / m_peer, j = e % m_peer;
     const int r = pr + (pr >= rank ? 1 : 0);
     peer_keys[e] = cluster.map_shared_rank(sorted, r)[j];
@@ -286,16 +286,16 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
   for (int li = tid; li < n_cand; li += kRankThreads) {
     const unsigned long long key = sorted[li];
     int rk = li;
-    int pos[kRankCluster - 1];                            // number of each peer's codes below key; the seven
+    int pos[CL - 1];                            // number of each peer's codes below key; the
 #pragma unroll                                            // branch-free searches run side by side
-    for (int pr = 0; pr < kRankCluster - 1; ++pr) pos[pr] = 0;
+    for (int pr = 0; pr < CL - 1; ++pr) pos[pr] = 0;
     for (int step = m_peer >> 1; step > 0; step >>= 1) {
 #pragma unroll
-      for (int pr = 0; pr < kRankCluster - 1; ++pr)
+      for (int pr = 0; pr < CL - 1; ++pr)
         pos[pr] += peer_keys[(size_t)pr * m_peer + pos[pr] + step - 1] < key ? step : 0;
     }
 #pragma unroll
-    for (int pr = 0; pr < kRankCluster - 1; ++pr) {
+    for (int pr = 0; pr < CL - 1; ++pr) {
       pos[pr] += peer_keys[(size_t)pr * m_peer + pos[pr]] < key ? 1 : 0;
       rk += pos[pr];
     }
@@ -361,28 +361,37 @@ __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, con
   store_vec<T, NE>(qbar + warp * D + lane * NE, acc);
 }
 
-template <typename T, int D>
+template <typename T, int D, int CL>
 static cudaError_t launch_rank_t(const DevParams& P, const void* q, int32_t* q_idx, cudaStream_t st) {
   constexpr int LG = D / 8, RPI = kRankThreads / LG;
-  int rpc = (P.chunk + kRankCluster - 1) / kRankCluster;
+  int rpc = (P.chunk + CL - 1) / CL;
   int n_sort = 32;
   while (n_sort < rpc) n_sort <<= 1;
   const size_t row_bytes = (size_t)rpc * D * sizeof(T);
   int m_peer = 1;
   while (m_peer < P.n_sel && m_peer < n_sort) m_peer <<= 1;
-  const size_t fixed = (size_t)n_sort * 16 + (size_t)RPI * D * 4 + (size_t)((rpc + 3) & ~3) * 4 + (((size_t)(kRankCluster - 1) * m_peer + 1) & ~(size_t)1) * 8;
+  const size_t fixed = (size_t)n_sort * 16 + (size_t)RPI * D * 4 + (size_t)((rpc + 3) & ~3) * 4 + (((size_t)(CL - 1) * m_peer + 1) & ~(size_t)1) * 8;
   const int staged = fixed + row_bytes <= kRankStageLimit + 48 * 1024 && row_bytes <= kRankStageLimit ? 1 : 0;
   const size_t smem = fixed + (staged ? row_bytes : 0);
-  cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_kernel(rank_queries_kernel<T, D>, dim3(P.batch * P.n_q * kRankCluster), dim3(kRankThreads), smem, st, kRankCluster,
-                       false, P, (const T*)q, q_idx, rpc, n_sort, staged, m_peer);
+  return launch_kernel(rank_queries_kernel<T, D, CL>, dim3(P.batch * P.n_q * CL), dim3(kRankThreads), smem, st, CL, false, P,
+                       (const T*)q, q_idx, rpc, n_sort, staged, m_peer);
+}
+
+// A cluster per (sequence, head), sized so that a CTA's slice is about 256 rows: shorter slices only multiply the
+// per-CTA costs (four cluster barriers, the sort, the merge).
+template <typename T, int D>
+static cudaError_t launch_rank_d(const DevParams& P, const void* q, int32_t* q_idx, cudaStream_t st) {
+  if (P.chunk <= 512) return launch_rank_t<T, D, 2>(P, q, q_idx, st);
+  if (P.chunk <= 1024) return launch_rank_t<T, D, 4>(P, q, q_idx, st);
+  return launch_rank_t<T, D, kRankCluster>(P, q, q_idx, st);
 }
 
 cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st) {
   cudaError_t e;
-  if (dtype == QUOKA_BF16) e = P.d == 128 ? launch_rank_t<__nv_bfloat16, 128>(P, q, q_idx, st) : launch_rank_t<__nv_bfloat16, 64>(P, q, q_idx, st);
-  else e = P.d == 128 ? launch_rank_t<float, 128>(P, q, q_idx, st) : launch_rank_t<float, 64>(P, q, q_idx, st);
+  if (dtype == QUOKA_BF16) e = P.d == 128 ? launch_rank_d<__nv_bfloat16, 128>(P, q, q_idx, st) : launch_rank_d<__nv_bfloat16, 64>(P, q, q_idx, st);
+  else e = P.d == 128 ? launch_rank_d<float, 128>(P, q, q_idx, st) : launch_rank_d<float, 64>(P, q, q_idx, st);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
