@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
       const int rc = max(min(r, n_loc - 1), 0);              // clamped (an empty slice reads row 0 / the last row)
       const uint4* grow = reinterpret_cast<const uint4*>(qh + (long long)min(lo + rc, C - 1) * P.q_st);
       float dot = 0.f, nn = 0.f;
-#pragma unroll
+#pragma unroll 4      // all eight words at once made the compiler spill
       for (int i = 0; i < HW; ++i) {
         const int c = half * HW + i;
         uint4 wv;
