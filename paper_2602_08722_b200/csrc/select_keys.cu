@@ -8,11 +8,12 @@
 //
 // select_keys_reg_kernel (the default): one CTA of 1024 threads per (sequence, KV head), or a cluster
 // of 2/4/8 CTAs for long rows, holds the whole row as order codes IN REGISTERS (up to 32 per thread:
-// the scores are read from memory exactly once, coalesced).  Three passes of 12 + 12 + 8 bits: each
-// pass histograms only the rows still matching the prefix with shared-memory atomics (a warp whose
-// lanes all carry the same digit adds once), the bin holding the B-th largest is found with a block-wide
-// suffix scan, and with a cluster the per-CTA histograms and counts are summed through distributed
-// shared memory.
+// the scores are read from memory exactly once, coalesced).  The digits are those of (code - smallest
+// code of the row) shifted up to the top bit, so that a row of similar scores still spreads over the
+// bins.  Three passes of 12 + 12 + 8 bits: each pass histograms only the rows still matching the prefix
+// with shared-memory atomics, the bin holding the B-th largest is found with a block-wide suffix scan,
+// and with a cluster the per-CTA histograms and counts are summed through distributed shared memory.
+// The list is collected in shared memory and copied out with full-width stores (single CTA).
 // select_keys_kernel (one CTA per head, scores re-read from L2 every pass, 8-bit digits) serves rows
 // too long for that.
 #include <cooperative_groups.h>

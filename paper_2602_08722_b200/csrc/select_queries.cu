@@ -56,12 +56,11 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
   constexpr int RPI = kRankThreads / LG;    // rows per iteration
   constexpr int NW = sizeof(T) * 8 / 16;    // 16-byte words per lane
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // dynamic shared memory: sort keys | reduction buffer | (unused) | peer codes | staged rows
+  // dynamic shared memory: sort keys | reduction buffer | peer codes | staged rows
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);               // [n_sort] 32-key sorted runs
   unsigned long long* sorted = keys + n_sort;                                               // [n_sort] the sorted slice
   float* red = reinterpret_cast<float*>(smem_raw + (size_t)n_sort * 16);                    // [RPI][D]
-  float* norms = red + RPI * D;                                                             // [rpc]
-  unsigned long long* peer_keys = reinterpret_cast<unsigned long long*>(norms + ((rpc + 3) & ~3));   // [7][m_peer]
+  unsigned long long* peer_keys = reinterpret_cast<unsigned long long*>(red + RPI * D);     // [CL - 1][m_peer]
   uint4* rows = reinterpret_cast<uint4*>(peer_keys + (((size_t)(CL - 1) * m_peer + 1) & ~(size_t)1));   // [rpc][LG][NW]
   __shared__ float part[D];                 // this CTA's share of the column sums
   __shared__ __align__(16) float M[D];
@@ -370,7 +369,7 @@ static cudaError_t launch_rank_t(const DevParams& P, const void* q, int32_t* q_i
   const size_t row_bytes = (size_t)rpc * D * sizeof(T);
   int m_peer = 1;
   while (m_peer < P.n_sel && m_peer < n_sort) m_peer <<= 1;
-  const size_t fixed = (size_t)n_sort * 16 + (size_t)RPI * D * 4 + (size_t)((rpc + 3) & ~3) * 4 + (((size_t)(CL - 1) * m_peer + 1) & ~(size_t)1) * 8;
+  const size_t fixed = (size_t)n_sort * 16 + (size_t)RPI * D * 4 + (((size_t)(CL - 1) * m_peer + 1) & ~(size_t)1) * 8;
   const int staged = fixed + row_bytes <= kRankStageLimit + 48 * 1024 && row_bytes <= kRankStageLimit ? 1 : 0;
   const size_t smem = fixed + (staged ? row_bytes : 0);
   cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
