@@ -115,7 +115,6 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtx wc{&abort_flag, P.status};
-  grid_launch_dependents();                  // the selection kernel may become resident; it waits for this grid itself
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -132,6 +131,10 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Only now may the kernels after this one become resident (the selection kernel, and through it the attention
+  // kernel, which also allocates tensor memory): every CTA of this grid holds its tensor memory by then, so a
+  // later grid can never take the columns a CTA of this one still has to wait for.
+  grid_launch_dependents();
 
   const long long total = total_tiles(P);
   const long long lo = total * blockIdx.x / gridDim.x, hi = total * (blockIdx.x + 1) / gridDim.x;
