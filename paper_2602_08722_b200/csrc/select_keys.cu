@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_kernel(DevParams P, c
 
 constexpr int kRegBins = 4096;            // 12-bit digits
 constexpr int kHistWords = 2 * kRegBins + 256;
+constexpr int kCandMax = 256;              // rows of the threshold's bin that are listed instead of passed again
 
 // Warp w of CTA r owns positions [r*1024*ITEMS + w*32*ITEMS, +32*ITEMS); lane l holds i*32 + l of them.
 template <int ITEMS, int CL>
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
                                                                        int32_t* __restrict__ k_idx,
                                                                        int32_t* __restrict__ k_cnt) {
   __shared__ uint32_t hist_all[kHistWords];     // one histogram per pass, zeroed once: no barrier to re-use one
-  __shared__ uint32_t s_prefix, s_need;
+  __shared__ uint32_t s_prefix, s_need, s_cand, s_n;
   __shared__ uint32_t warp_val[32];
   __shared__ uint32_t warp_off[33];
   __shared__ uint32_t cta_cnt[2];               // rows of this CTA above / equal to the threshold
@@ -176,6 +177,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     cmax = max(cmax, c);
   }
   for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
+  if (tid == 0) s_n = 0;
   // The codes of one row of scores share their leading bits (cosines of similar size): digits of the raw code
   // would put most rows into a few bins, which serialises the shared-memory atomics and leaves every pass
   // with many rows.  The digits are taken from (code - smallest code) shifted up to the top bit instead; the map
@@ -208,8 +210,6 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
     const int nb = pass == 2 ? 256 : kRegBins;
     uint32_t* hist = hist_all + pass * kRegBins;
-    // (compacting the threshold bin's rows into a list for the later passes was tried: building the list
-    // costs as much as the two passes it shortens)
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
       const bool live = (base + 32 * i < T) && ((code[i] & mask) == prefix);
@@ -259,6 +259,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
         if (cum + c[k] >= need) {
           s_prefix = prefix | ((uint32_t)(nb - 1 - (4 * tid + k)) << shift);
           s_need = need - cum;
+          s_cand = c[k];
           break;
         }
         cum += c[k];
@@ -268,6 +269,33 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     prefix = s_prefix;
     need = s_need;
     mask |= (uint32_t)(nb - 1) << shift;
+    // With the digits spread over the row's own range the first pass usually leaves a handful of rows in the
+    // threshold's bin.  A single CTA then lists them (over the second pass's histogram, which it will not need)
+    // and finds the `need`-th largest among them directly: every listed row counts the listed rows above and
+    // equal to it.  More rows than the list holds (many equal scores): the remaining digit passes run instead.
+    if (CL == 1 && pass == 0 && s_cand <= (uint32_t)kCandMax) {
+      const uint32_t n_cand = s_cand;
+      uint32_t* cand = hist_all + kRegBins;
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i) {
+        if ((base + 32 * i < T) && ((code[i] & mask) == prefix)) cand[atomicAdd(&s_n, 1u)] = code[i];
+      }
+      __syncthreads();
+      if ((uint32_t)tid < n_cand) {
+        const uint32_t my = cand[tid];
+        uint32_t g = 0, e = 0;
+        for (uint32_t j = 0; j < n_cand; ++j) {
+          const uint32_t c2 = cand[j];
+          g += c2 > my ? 1u : 0u;
+          e += c2 == my ? 1u : 0u;
+        }
+        if (g < need && need <= g + e) { s_prefix = my; s_need = need - g; }     // equal rows write the same values
+      }
+      __syncthreads();
+      prefix = s_prefix;
+      need = s_need;
+      break;
+    }
   }
   // prefix = (shifted) code of the B-th largest score.  Rows at or above it, per warp and before each warp:
   const uint32_t thr = prefix;
