@@ -8,12 +8,13 @@
 //
 // select_keys_reg_kernel (the default): one CTA of 1024 threads per (sequence, KV head), or a cluster
 // of 2/4/8 CTAs for long rows, holds the whole row as order codes IN REGISTERS (up to 32 per thread:
-// the scores are read from memory exactly once, coalesced).  The digits are those of (code - smallest
-// code of the row) shifted up to the top bit, so that a row of similar scores still spreads over the
-// bins.  Three passes of 12 + 12 + 8 bits: each pass histograms only the rows still matching the prefix
-// with shared-memory atomics, the bin holding the B-th largest is found with a block-wide suffix scan,
-// and with a cluster the per-CTA histograms and counts are summed through distributed shared memory.
-// The list is collected in shared memory and copied out with full-width stores (single CTA).
+// the scores are read from memory exactly once, coalesced).  A single CTA first histograms the row over
+// bins linear in the score, finds the bin of the B-th largest with a block-wide suffix scan, and ranks
+// that bin's few rows against each other.  Otherwise (clusters; many equal scores) three digit passes of
+// 12 + 12 + 8 bits over (code - smallest code of the row) shifted up to the top bit: each pass histograms
+// only the rows still matching the prefix, and with a cluster the per-CTA histograms and counts are
+// summed through distributed shared memory.  The list is collected in shared memory and copied out with
+// full-width stores (single CTA).
 // select_keys_kernel (one CTA per head, scores re-read from L2 every pass, 8-bit digits) serves rows
 // too long for that.
 #include <cooperative_groups.h>
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
                                                                        int32_t* __restrict__ k_idx,
                                                                        int32_t* __restrict__ k_cnt) {
   __shared__ uint32_t hist_all[kHistWords];     // one histogram per pass, zeroed once: no barrier to re-use one
-  __shared__ uint32_t s_prefix, s_need, s_cand, s_n;
+  __shared__ uint32_t s_bin, s_need, s_cand, s_n;
   __shared__ uint32_t warp_val[32];
   __shared__ uint32_t warp_off[33];
   __shared__ uint32_t cta_cnt[2];               // rows of this CTA above / equal to the threshold
@@ -178,10 +179,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   }
   for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
   if (tid == 0) s_n = 0;
-  // The codes of one row of scores share their leading bits (cosines of similar size): digits of the raw code
-  // would put most rows into a few bins, which serialises the shared-memory atomics and leaves every pass
-  // with many rows.  The digits are taken from (code - smallest code) shifted up to the top bit instead; the map
-  // keeps the order, and no bit is lost.
+  // smallest and largest code of the row
   cmin = __reduce_min_sync(0xFFFFFFFFu, cmin);
   cmax = __reduce_max_sync(0xFFFFFFFFu, cmax);
   if (lane == 0) { warp_val[wid] = cmin; warp_off[wid] = cmax; }
@@ -199,24 +197,11 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     }
     cluster.sync();                                // cta_cnt is used again below
   }
-  const int up = min(__clz((int)(cmax - cmin)), 31);
-#pragma unroll
-  for (int i = 0; i < ITEMS; ++i) code[i] = (code[i] - cmin) << up;
-  __syncthreads();                                 // the histograms are zero, warp_val / warp_off free again
   const uint32_t lt = (1u << lane) - 1u;
-  uint32_t prefix = 0, mask = 0, need = (uint32_t)B;
-#pragma unroll 1
-  for (int pass = 0; pass < 3; ++pass) {
-    const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
-    const int nb = pass == 2 ? 256 : kRegBins;
-    uint32_t* hist = hist_all + pass * kRegBins;
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) {
-      const bool live = (base + 32 * i < T) && ((code[i] & mask) == prefix);
-      if (live) atomicAdd(&hist[(code[i] >> shift) & (uint32_t)(nb - 1)], 1u);
-    }
-    if (CL > 1) cluster.sync(); else __syncthreads();
-    // thread t owns the 4 bins nb-1-4t .. nb-4-4t (descending); find where the running count reaches `need`
+  uint32_t prefix = 0, need = (uint32_t)B;
+  // Finds the bin (counted from the top) in which the running count reaches `need`: thread t owns the 4 bins
+  // nb-1-4t .. nb-4-4t; leaves the bin in s_bin, what is still needed inside it in s_need, its size in s_cand.
+  const auto find_bin = [&](uint32_t* hist, int nb) {
     uint32_t c[4] = {0, 0, 0, 0}, sum = 0;
     if (4 * tid < nb) {
       if (CL > 1) {
@@ -257,7 +242,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         if (cum + c[k] >= need) {
-          s_prefix = prefix | ((uint32_t)(nb - 1 - (4 * tid + k)) << shift);
+          s_bin = (uint32_t)(nb - 1 - (4 * tid + k));
           s_need = need - cum;
           s_cand = c[k];
           break;
@@ -266,20 +251,31 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
       }
     }
     __syncthreads();
-    prefix = s_prefix;
-    need = s_need;
-    mask |= (uint32_t)(nb - 1) << shift;
-    // With the digits spread over the row's own range the first pass usually leaves a handful of rows in the
-    // threshold's bin.  A single CTA then lists them (over the second pass's histogram, which it will not need)
-    // and finds the `need`-th largest among them directly: every listed row counts the listed rows above and
-    // equal to it.  More rows than the list holds (many equal scores): the remaining digit passes run instead.
-    if (CL == 1 && pass == 0 && s_cand <= (uint32_t)kCandMax) {
-      const uint32_t n_cand = s_cand;
+  };
+  bool found = false;
+  int up = 0;                                      // the codes are compared as (code - sub) << up: raw unless the digit
+  uint32_t sub = 0;                                // passes ran
+  if (CL == 1) {
+    // ---- Single CTA, first try: ONE histogram over 4096 bins that are linear in the score between the row's
+    // smallest and largest (a monotone map, so the bin of the B-th largest holds it).  A row of cosines then
+    // leaves a few dozen rows in that bin; they are listed (over the second histogram's words) and every listed
+    // row counts the listed rows above and equal to it, which gives the exact code of the B-th largest.
+    const float fmin = order_key_to_float(cmin), fmax = order_key_to_float(cmax);
+    const float scale = fmax > fmin ? (float)kRegBins / (fmax - fmin) : 0.f;
+    const auto bin_of = [&](uint32_t c) { return min(kRegBins - 1, (int)((order_key_to_float(c) - fmin) * scale)); };
+    __syncthreads();                               // the histograms are zero, warp_val / warp_off free again
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i)
+      if (base + 32 * i < T) atomicAdd(&hist_all[bin_of(code[i])], 1u);
+    __syncthreads();
+    find_bin(hist_all, kRegBins);
+    if (s_cand <= (uint32_t)kCandMax) {
+      const uint32_t n_cand = s_cand, bin = s_bin;
+      need = s_need;
       uint32_t* cand = hist_all + kRegBins;
 #pragma unroll
-      for (int i = 0; i < ITEMS; ++i) {
-        if ((base + 32 * i < T) && ((code[i] & mask) == prefix)) cand[atomicAdd(&s_n, 1u)] = code[i];
-      }
+      for (int i = 0; i < ITEMS; ++i)
+        if (base + 32 * i < T && (uint32_t)bin_of(code[i]) == bin) cand[atomicAdd(&s_n, 1u)] = code[i];
       __syncthreads();
       if ((uint32_t)tid < n_cand) {
         const uint32_t my = cand[tid];
@@ -289,15 +285,47 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
           g += c2 > my ? 1u : 0u;
           e += c2 == my ? 1u : 0u;
         }
-        if (g < need && need <= g + e) { s_prefix = my; s_need = need - g; }     // equal rows write the same values
+        if (g < need && need <= g + e) { s_bin = my; s_need = need - g; }       // equal rows write the same values
       }
       __syncthreads();
-      prefix = s_prefix;
+      prefix = s_bin;
       need = s_need;
-      break;
+      found = true;
+    } else {
+      // many equal scores: start over with the digit passes below
+      for (int i = tid; i < kRegBins; i += kSelThreads) hist_all[i] = 0;
+      need = (uint32_t)B;
     }
   }
-  // prefix = (shifted) code of the B-th largest score.  Rows at or above it, per warp and before each warp:
+  if (!found) {
+    // ---- Digit passes 12 + 12 + 8 bits, most significant first.  The codes of one row of scores share their leading
+    // bits: the digits are taken from (code - smallest code) shifted up to the top bit, a map that keeps the order
+    // and loses no bit.
+    up = min(__clz((int)(cmax - cmin)), 31);
+    sub = cmin;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) code[i] = (code[i] - sub) << up;
+    __syncthreads();                               // the histograms are zero, warp_val / warp_off free again
+    uint32_t mask = 0;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
+      const int nb = pass == 2 ? 256 : kRegBins;
+      uint32_t* hist = hist_all + pass * kRegBins;
+#pragma unroll
+      for (int i = 0; i < ITEMS; ++i) {
+        const bool live = (base + 32 * i < T) && ((code[i] & mask) == prefix);
+        if (live) atomicAdd(&hist[(code[i] >> shift) & (uint32_t)(nb - 1)], 1u);
+      }
+      if (CL > 1) cluster.sync(); else __syncthreads();
+      find_bin(hist, nb);
+      prefix |= s_bin << shift;
+      need = s_need;
+      mask |= (uint32_t)(nb - 1) << shift;
+    }
+  }
+  // prefix = code of the B-th largest score (shifted, if the digit passes ran).  Rows at or above it, per warp and
+  // before each warp:
   const uint32_t thr = prefix;
   uint32_t w_ge = 0;
 #pragma unroll
@@ -356,7 +384,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll 1
     for (int i = 0; i < ITEMS; ++i) {
       const int pos = base + 32 * i;
-      const uint32_t c = (float_order_key(__ldcg(row + min(pos, T - 1))) - cmin) << up;
+      const uint32_t c = (float_order_key(__ldcg(row + min(pos, T - 1))) - sub) << up;
       w_gt += (pos < T && c > thr) ? 1u : 0u;
       w_eq += (pos < T && c == thr) ? 1u : 0u;
     }
@@ -389,7 +417,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 #pragma unroll 1
     for (int i = 0; i < ITEMS; ++i) {
       const int pos = base + 32 * i;
-      const uint32_t c = (float_order_key(__ldcg(row + min(pos, T - 1))) - cmin) << up;
+      const uint32_t c = (float_order_key(__ldcg(row + min(pos, T - 1))) - sub) << up;
       const bool gt = pos < T && c > thr, eq = pos < T && c == thr;
       const uint32_t b_gt = __ballot_sync(0xFFFFFFFFu, gt), b_eq = __ballot_sync(0xFFFFFFFFu, eq);
       const uint32_t gt_before = run_gt + (uint32_t)__popc(b_gt & lt);
