@@ -179,7 +179,7 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 // ---- launch functions implemented in the .cu files (host side) -------------------------------
 // `chained`: the kernel before it on the stream is the one of the same fused call whose output it reads (see above).
 cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st);
-cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, const int32_t* q_idx, void* qbar,
+cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, void* qbar,
                                      cudaStream_t st, bool chained = false);
 cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,
                                    cudaStream_t st);

@@ -74,11 +74,7 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
   int32_t* out = q_idx + (long long)head * N;
   const int tid = threadIdx.x;
 
-  if (C <= P.n_retain) {                    // no sub-selection: every query, in position order
-    for (int j = rank * kRankThreads + tid; j < C; j += CL * kRankThreads) out[j] = j;
-    return;
-  }
-
+  // (C <= N_Q, where every query is kept, never reaches this kernel: the aggregation kernel writes those ranks)
   const T* qh = q + (long long)s * P.q_sb + (long long)h * P.q_sh;
   const int lane_in_row = tid % LG;
   const int row_slot = tid / LG;
@@ -305,10 +301,13 @@ __global__ void __launch_bounds__(kRankThreads, 2) rank_queries_kernel(DevParams
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, const T* __restrict__ q,
-                                                                 const int32_t* __restrict__ q_idx,
+                                                                 int32_t* __restrict__ q_idx,
                                                                  T* __restrict__ qbar) {
   grid_launch_dependents();
   grid_dependency_wait();                   // the ranks come from the kernel before
+  // a chunk no longer than the number of retained queries keeps every query, in position order (Alg. 1's `if`):
+  // no ranking kernel runs then, and this kernel writes the identity ranks itself
+  const bool identity = P.chunk <= P.n_retain;
   constexpr int NE = D / 32;
   const int N = P.n_sel;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -324,7 +323,11 @@ __global__ void __launch_bounds__(256) aggregate_queries_kernel(DevParams P, con
   for (int g0 = 0; g0 < P.group; g0 += 32) {
     // the group's ranks in one load, then the rows four at a time so their loads overlap
     const int gl = g0 + lane;
-    const int r_lane = gl < P.group ? __ldcg(q_idx + ((int64_t)s * P.n_q + kv * P.group + gl) * N + j) : 0;
+    int r_lane = j;
+    if (gl < P.group) {
+      int32_t* slot = q_idx + ((int64_t)s * P.n_q + kv * P.group + gl) * N + j;
+      if (identity) *slot = j; else r_lane = __ldcg(slot);
+    }
     const int g_end = min(32, P.group - g0);
     for (int g4 = 0; g4 < g_end; g4 += 4) {
       float x[4][NE];
@@ -388,6 +391,7 @@ static cudaError_t launch_rank_d(const DevParams& P, const void* q, int32_t* q_i
 }
 
 cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, cudaStream_t st) {
+  if (P.chunk <= P.n_retain) return cudaSuccess;      // every query is kept: the aggregation kernel writes the ranks
   cudaError_t e;
   if (dtype == QUOKA_BF16) e = P.d == 128 ? launch_rank_d<__nv_bfloat16, 128>(P, q, q_idx, st) : launch_rank_d<__nv_bfloat16, 64>(P, q, q_idx, st);
   else e = P.d == 128 ? launch_rank_d<float, 128>(P, q, q_idx, st) : launch_rank_d<float, 64>(P, q, q_idx, st);
@@ -395,7 +399,7 @@ cudaError_t launch_rank_queries(const DevParams& P, int dtype, const void* q, in
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, const int32_t* q_idx, void* qbar,
+cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* q, int32_t* q_idx, void* qbar,
                                      cudaStream_t st, bool chained) {
   const int64_t warps = (int64_t)P.batch * P.n_kv * P.n_sel;
   const dim3 grid((unsigned)((warps * 32 + 255) / 256)), block(256);
