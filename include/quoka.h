@@ -173,7 +173,11 @@ quoka_status quoka_dense_chunk_attn(const quoka_params* p, const void* q, const 
 
 /* Alg. 2, loop body: the four steps above on `stream` with the intermediates in
  * the workspace.  k_idx_out ([b][n_KV][cap]) and k_cnt_out ([b]) may be NULL; when
- * given they receive the selection that was used. */
+ * given they receive the selection that was used.  The kernels of one call are
+ * launched so that each may become resident while the one before it still runs
+ * (each waits for its producer itself); towards everything else on `stream` the
+ * call is ordered like a single kernel: it starts after the work before it and
+ * the work after it starts when its last kernel has completed. */
 quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
                                  void* out, int32_t* k_idx_out, int32_t* k_cnt_out,
                                  void* ws, size_t ws_bytes, void* stream);
