@@ -147,7 +147,6 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   __shared__ uint32_t cta_cnt[2];               // rows of this CTA above / equal to the threshold
 
   grid_launch_dependents();     // the attention kernel may start now: it waits for this grid itself before it reads the list
-  grid_dependency_wait();       // the scores come from the kernel before
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = CL > 1 ? (int)cluster.block_rank() : 0;
   const int head = blockIdx.x / CL;
@@ -167,6 +166,11 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     return;
   }
   const int base = (rank * kSelThreads + wid * 32) * ITEMS + lane;      // position of item i: base + 32 i
+  for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
+  if (tid == 0) s_n = 0;
+  // Everything above needs nothing from the kernel before this one (launched early, it has run under that kernel's
+  // tail); the scores do.
+  grid_dependency_wait();
   uint32_t code[ITEMS];
   uint32_t cmin = 0xFFFFFFFFu, cmax = 0u;
 #pragma unroll
@@ -177,8 +181,6 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
     cmin = min(cmin, c);
     cmax = max(cmax, c);
   }
-  for (int i = tid; i < kHistWords; i += kSelThreads) hist_all[i] = 0;
-  if (tid == 0) s_n = 0;
   // smallest and largest code of the row
   cmin = __reduce_min_sync(0xFFFFFFFFu, cmin);
   cmax = __reduce_max_sync(0xFFFFFFFFu, cmax);
