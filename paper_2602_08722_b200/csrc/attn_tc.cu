@@ -236,17 +236,20 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
       const int lim = visible_cols(tile_rows<SPARSE>(g, t), row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
       // ---- pass 1: the row maximum.  All four 32-column loads are issued together (one tensor-memory round
-      // trip); the row is read once more, in 64-key blocks, by pass 2: tensor memory is cheap to re-read, and
-      // not keeping the 128 values live leaves pass 2 the registers for a whole block of exponentials in flight.
+      // trip).  The first 64 scores stay in registers for pass 2, the other 64 are read once more there: keeping
+      // 96 or all 128 alive next to a block of exponentials in flight does not fit the 168 registers (it spills).
       float mx;
+      uint32_t v0[64];                                         // the first 64 scores stay in registers for pass 2
       {
-        uint32_t c0[32], c1[32], c2[32], c3[32];
-        tmem_ld32(s_addr, c0);
-        tmem_ld32(s_addr + 32, c1);
+        uint32_t c2[32], c3[32];
+        tmem_ld32(s_addr, v0);
+        tmem_ld32(s_addr + 32, v0 + 32);
         tmem_ld32(s_addr + 64, c2);
         tmem_ld32(s_addr + 96, c3);
         tmem_wait_ld();
-        mx = fmaxf(fmaxf(max32(c0, masked, 0, lim), max32(c1, masked, 32, lim)),
+        uint32_t (&a0)[32] = *reinterpret_cast<uint32_t (*)[32]>(v0);
+        uint32_t (&a1)[32] = *reinterpret_cast<uint32_t (*)[32]>(v0 + 32);
+        mx = fmaxf(fmaxf(max32(a0, masked, 0, lim), max32(a1, masked, 32, lim)),
                    fmaxf(max32(c2, masked, 64, lim), max32(c3, masked, 96, lim)));
       }
       const float m_tile = mx * scale_log2;
@@ -279,12 +282,17 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t v[64], pk[32];
-        tmem_ld32(s_addr + half * 64, v);
-        tmem_ld32(s_addr + half * 64 + 32, v + 32);
-        tmem_wait_ld();
-        if (masked) {
+        if (half == 0) {
 #pragma unroll
-          for (int i = 0; i < 64; ++i) if (half * 64 + i >= lim) v[i] = 0xFF800000u;   // -inf: exp2 gives exactly 0
+          for (int i = 0; i < 64; ++i) v[i] = v0[i];          // masked already by pass 1
+        } else {
+          tmem_ld32(s_addr + 64, v);
+          tmem_ld32(s_addr + 96, v + 32);
+          tmem_wait_ld();
+          if (masked) {
+#pragma unroll
+            for (int i = 0; i < 64; ++i) if (64 + i >= lim) v[i] = 0xFF800000u;   // -inf: exp2 gives exactly 0
+          }
         }
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
