@@ -32,7 +32,7 @@ METRIC = "us_per_prefill_chunk"
 UNIT = "us"
 # DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu capture of that workload
 # (profiles/kernels_full_<workload>.md); None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {("llama8b_32k", "sparse_attn"): 42.4e6}
+NCU_TRAFFIC_BYTES = {("llama8b_32k", "sparse_attn"): 42.5e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
