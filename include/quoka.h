@@ -59,7 +59,8 @@ typedef enum {
   QUOKA_ERR_WORKSPACE = 3,    /* workspace pointer null / misaligned / smaller than quoka_workspace_size */
   QUOKA_ERR_CUDA = 4,         /* a CUDA runtime or driver call failed (launch, tensor-map encode) */
   QUOKA_ERR_TIMEOUT = 5,      /* device status word: a bounded wait inside a kernel ran out */
-  QUOKA_ERR_STATIC_LIMIT = 6  /* quoka_prefill_chunk_static: the problem needs more scratch than the built-in array */
+  QUOKA_ERR_STATIC_LIMIT = 6, /* quoka_prefill_chunk_static: the problem needs more scratch than the built-in array */
+  QUOKA_ERR_BAD_INDEX = 7     /* device status word (debug build): a selected row or a page id was out of range */
 } quoka_status;
 
 typedef enum { QUOKA_BF16 = 0, QUOKA_F32 = 1 } quoka_dtype;
@@ -194,6 +195,14 @@ quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_
                                       void* out_host, void* q_dev, void* k_cache, void* v_cache, void* out_dev,
                                       void* ws, size_t ws_bytes, void* stream);
 
+/* Alg. 2, "append K_i, V_i to the cache": copies the chunk's keys and values, dense [b][n_KV][C][d] in DEVICE
+ * memory, into rows [T_s, T_s + C) of the cache (contiguous by strides, or paged through the block table), with
+ * T_s read from p->ctx_len on the device.  Call it before the chunk's quoka_prefill_chunk (see "Cache layout").
+ * When k_inv_norm is not NULL the inverse norms of the appended rows are written as quoka_update_key_norms
+ * would.  The caller advances ctx_len by C after the chunk's attention. */
+quoka_status quoka_append_kv(const quoka_params* p, const void* k_new, const void* v_new, void* k_cache,
+                             void* v_cache, float* k_inv_norm, void* ws, size_t ws_bytes, void* stream);
+
 /* (The paper has no counterpart of this call: it is a deployment variant of quoka_prefill_chunk.)
  * The same loop body for callers that cannot allocate device memory and so have no workspace to
  * pass: a process whose KV-cache pool already owns all of HBM, or a latency-critical loop in which
@@ -210,21 +219,48 @@ quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_
  *     contents.  The status word is cleared at the start of every call; nothing else needs to start
  *     at zero.  Two calls whose work overlaps on the same GPU (different streams, or different host
  *     threads) race on the array: serialise them.
- *   - A timed-out device wait cannot be read back through quoka_last_device_status, which needs
- *     the workspace pointer; the outputs of such a call are undefined. */
+ *   - The array's status word is read (and cleared) with quoka_last_device_status(NULL, stream, &st);
+ *     read it before the next static call, which clears it.
+ *   - The array's address is looked up once per device and remembered: after cudaDeviceReset the
+ *     process must not use this entry point again. */
 #define QUOKA_STATIC_SCRATCH_BYTES (8u << 20)
 quoka_status quoka_prefill_chunk_static(const quoka_params* p, const void* q, const void* k_cache,
                                         const void* v_cache, void* out, int32_t* k_idx_out, int32_t* k_cnt_out,
                                         void* stream);
 
 /* Copies the device status word of `ws` to the host (synchronises `stream`) and
- * clears it.  *status_out is a quoka_status. */
+ * clears it.  *status_out is a quoka_status.  ws == NULL reads the status word of the built-in
+ * array that quoka_prefill_chunk_static uses on the current device.  After a QUOKA_ERR_TIMEOUT the
+ * outputs of the call that hit it are undefined (the kernel left its loops and ran its teardown
+ * with work possibly still outstanding). */
 quoka_status quoka_last_device_status(void* ws, void* stream, int32_t* status_out);
 
 const char* quoka_status_string(quoka_status s);
 
 /* Number of kernels this library has launched in this process (all entry points). */
 int64_t quoka_launch_count(void);
+
+/* ---- diagnostics (no counterpart in the paper) ------------------------------------------------
+ * QUOKA_LOG=1 in the environment prints one line per kernel launch (name, grid, block, dynamic
+ * shared memory, cluster width) on stderr.
+ *
+ * A build with -DQUOKA_DEBUG (python -m paper_2602_08722_b200.build --debug, libquoka_debug.so)
+ * range-checks every selected-row index and every block-table entry the attention kernel is about
+ * to use; a bad one records QUOKA_ERR_BAD_INDEX in the status word and the row is treated as
+ * absent (zero-filled, masked) instead of being read. */
+
+/* HOST-side check of a paged cache's block table before it is uploaded: ctx_len_host [batch] and
+ * block_table_host [batch][max_pages_per_seq] are HOST arrays.  Every page that rows
+ * [0, T_s + C) of a sequence need must lie inside the pool (0 <= page < kv_rows) and no physical
+ * page may be used twice.  Returns QUOKA_ERR_INVALID_ARG otherwise.  Launches nothing. */
+quoka_status quoka_check_block_table(const quoka_params* p, const int32_t* ctx_len_host,
+                                     const int32_t* block_table_host);
+
+/* Self-test of the bounded device wait: launches one warp that waits on a barrier nobody signals,
+ * with a limit of limit_cycles SM cycles (1 .. 2e9).  The wait must give up: *gave_up (DEVICE
+ * int32) becomes 1, the status word of `ws` becomes QUOKA_ERR_TIMEOUT, and the kernel returns.
+ * Exercises exactly the wait every tensor-core kernel of the library uses. */
+quoka_status quoka_selftest_wait_timeout(void* ws, int64_t limit_cycles, int32_t* gave_up, void* stream);
 
 #ifdef __cplusplus
 }

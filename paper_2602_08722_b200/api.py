@@ -15,7 +15,7 @@ import torch
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libquoka.so")
 _lib = None
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_STATIC_LIMIT = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_STATIC_LIMIT, ERR_BAD_INDEX = range(8)
 STATIC_SCRATCH_BYTES = 8 << 20
 BF16, F32 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TENSOR = 0, 1, 2
@@ -26,6 +26,7 @@ EXPORTS = [
     "quoka_kv_budget_cap", "quoka_workspace_size", "quoka_select_queries", "quoka_score_keys",
     "quoka_update_key_norms", "quoka_select_keys", "quoka_sparse_attn", "quoka_dense_chunk_attn", "quoka_prefill_chunk",
     "quoka_prefill_chunk_host", "quoka_prefill_chunk_static", "quoka_last_device_status", "quoka_status_string", "quoka_launch_count",
+    "quoka_append_kv", "quoka_check_block_table", "quoka_selftest_wait_timeout",
 ]
 
 
@@ -57,10 +58,22 @@ def load():
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(_LIB_PATH):
-        raise RuntimeError(f"{_LIB_PATH} is missing: the CUDA library has not been built "
+    _lib = _open(_LIB_PATH)
+    return _lib
+
+
+def open_debug_library():
+    """A second, independent handle: libquoka_debug.so (built with -DQUOKA_DEBUG).  Its functions are called
+    through ctypes directly (same argument types as load()'s); the functions of this module keep using libquoka.so."""
+    path = os.path.join(os.path.dirname(_LIB_PATH), "libquoka_debug.so")
+    return _open(path)
+
+
+def _open(path):
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: the CUDA library has not been built "
                            "(python -m paper_2602_08722_b200.build); there is no fallback path")
-    lib = C.CDLL(_LIB_PATH)
+    lib = C.CDLL(path)
     lib.quoka_status_string.restype = C.c_char_p
     lib.quoka_status_string.argtypes = [C.c_int]
     lib.quoka_launch_count.restype = C.c_int64
@@ -78,10 +91,12 @@ def load():
     lib.quoka_prefill_chunk_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.quoka_prefill_chunk_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp]
     lib.quoka_last_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+    lib.quoka_append_kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.quoka_check_block_table.argtypes = [pp, vp, vp]
+    lib.quoka_selftest_wait_timeout.argtypes = [vp, C.c_int64, vp, vp]
     for name in EXPORTS:
         if name not in ("quoka_status_string", "quoka_launch_count"):
             getattr(lib, name).restype = C.c_int
-    _lib = lib
     return lib
 
 
@@ -210,6 +225,21 @@ def quoka_last_device_status(ws, stream=None) -> int:
     st = C.c_int32(0)
     _check(load().quoka_last_device_status(_ptr(ws), _stream(stream), C.byref(st)), "quoka_last_device_status")
     return st.value
+
+
+def quoka_append_kv(p, k_new, v_new, k_cache, v_cache, k_inv_norm, ws, stream=None):
+    _check(load().quoka_append_kv(C.byref(p), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache),
+                                  _ptr(k_inv_norm), _ptr(ws), ws.numel(), _stream(stream)), "quoka_append_kv")
+
+
+def quoka_check_block_table(p, ctx_len_host, block_table_host) -> int:
+    """Status of the host-side block-table check (OK or ERR_INVALID_ARG); both arguments are CPU int32 tensors."""
+    return int(load().quoka_check_block_table(C.byref(p), _ptr(ctx_len_host), _ptr(block_table_host)))
+
+
+def quoka_selftest_wait_timeout(ws, limit_cycles, gave_up, stream=None):
+    _check(load().quoka_selftest_wait_timeout(_ptr(ws), int(limit_cycles), _ptr(gave_up), _stream(stream)),
+           "quoka_selftest_wait_timeout")
 
 
 def quoka_launch_count() -> int:

@@ -65,6 +65,7 @@ cudaError_t launch_attn_simt(const DevParams& P, int dtype, const void* q, const
                              const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st) {
   const int64_t warps = (int64_t)P.batch * P.n_q * P.chunk;
   const int grid = (int)((warps * 32 + 255) / 256);
+  log_launch("attn_simt", dim3(grid), dim3(256), 0, 1, false);
 #define QUOKA_ATTN(T_, D) \
   attn_simt_kernel<T_, D><<<grid, 256, 0, st>>>(P, (const T_*)q, (const T_*)k, (const T_*)v, k_idx, k_cnt, (T_*)out, lse)
   if (dtype == QUOKA_BF16) {

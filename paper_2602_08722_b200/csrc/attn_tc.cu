@@ -412,6 +412,12 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
           const int listed = __shfl_sync(0xFFFFFFFFu, t_list[(i * ROWS_PER_INSTR) / 32], (i * ROWS_PER_INSTR + rsub) & 31);
           t[i] = tr.from_list ? listed : (rr < tr.count ? tr.first + rr : -1);
         }
+#ifdef QUOKA_DEBUG
+        // debug build: a listed row outside [0, T) is recorded and treated as absent (zero-filled) instead of read
+#pragma unroll
+        for (int i = 0; i < RPT; ++i)
+          if (tr.from_list && (t[i] < -1 || t[i] >= g.T)) { atomicExch(P.status, (int32_t)QUOKA_ERR_BAD_INDEX); t[i] = -1; }
+#endif
         uint32_t off[RPT];
         if (P.page_size == 0) {
 #pragma unroll
@@ -420,7 +426,16 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 #pragma unroll
           for (int i = 0; i < RPT; ++i) {
             const int tc = max(t[i], 0);
-            off[i] = (uint32_t)__ldg(table + (tc >> 6)) * sb16 + base16 + (uint32_t)(tc & (kPage - 1)) * st16;
+            int page = __ldg(table + (tc >> 6));
+#ifdef QUOKA_DEBUG
+            // debug build: a page id outside the pool is recorded and the row treated as absent
+            if (t[i] >= 0 && (page < 0 || (long long)page >= P.kv_rows)) {
+              atomicExch(P.status, (int32_t)QUOKA_ERR_BAD_INDEX);
+              t[i] = -1;
+            }
+            if (page < 0 || (long long)page >= P.kv_rows) page = 0;
+#endif
+            off[i] = (uint32_t)page * sb16 + base16 + (uint32_t)(tc & (kPage - 1)) * st16;
           }
         }
 #pragma unroll
@@ -556,6 +571,7 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
   const size_t smem = 1024 + (2 + kSlots) * tile + 512;
   dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.batch);
   const bool sparse = k_idx != nullptr;
+  log_launch(sparse ? "attn_tc<sparse>" : "attn_tc<dense>", grid, dim3(kAttnThreads), smem, 1, sparse && after_selection);
   cudaError_t e = cudaSuccess;
   // Inside the fused call the sparse kernel is launched with programmatic stream serialisation: it may start
   // while the kernel before it on the stream (the key selection, which signals early and writes none of this

@@ -149,9 +149,12 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Launch with optional thread-block cluster width and, if `chained`, programmatic stream serialisation.
+void log_launch(const char* kernel, dim3 grid, dim3 block, size_t smem, int cluster, bool chained);
+
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                                 int cluster, bool chained, Args&&... args) {
+inline cudaError_t launch_kernel(const char* name, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, int cluster, bool chained, Args&&... args) {
+  log_launch(name, grid, block, smem, cluster, chained);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -190,6 +193,18 @@ cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t*
 cudaError_t launch_attn_simt(const DevParams& P, int dtype, const void* q, const void* k, const void* v,
                              const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st);
 
+cudaError_t launch_append_kv(const DevParams& P, int dtype, const void* k_new, const void* v_new, void* k_cache,
+                             void* v_cache, cudaStream_t st);
+
+// Host checks shared by the fused entry points (everything but the workspace); nothing is enqueued before they pass.
+quoka_status check_prefill_args(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                                const void* out);
+// Device address of the built-in scratch array on the current device (looked up once per device).
+quoka_status static_scratch_for_current_device(void** out);
+
 void count_launch(int n = 1);
+// QUOKA_LOG=1 in the environment: one line per kernel launch (grid, block, shared memory) on stderr.
+bool log_enabled();
+void log_launch(const char* kernel, dim3 grid, dim3 block, size_t smem, int cluster, bool chained);
 
 }  // namespace quoka

@@ -20,8 +20,10 @@ static std::mutex g_setup_mutex;
 static void* g_scratch_addr[kMaxDevices] = {};
 
 // The array's name is only a host-side handle; the address kernels can use has to be asked for,
-// once per device, with that device current.
-static quoka_status static_scratch_for_current_device(void** out) {
+// once per device, with that device current.  The address is remembered for the life of the
+// process: after cudaDeviceReset (or any teardown of the device's primary context) it is stale,
+// and this entry point must not be used again in that process.
+quoka_status static_scratch_for_current_device(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return QUOKA_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_setup_mutex);
@@ -39,9 +41,11 @@ static quoka_status static_scratch_for_current_device(void** out) {
 extern "C" quoka_status quoka_prefill_chunk_static(const quoka_params* p, const void* q, const void* k_cache,
                                                    const void* v_cache, void* out, int32_t* k_idx_out,
                                                    int32_t* k_cnt_out, void* stream) {
-  size_t need = 0;
-  quoka_status st = quoka_workspace_size(p, &need);
+  // every host-side refusal comes before the first thing put on the stream (the memset below)
+  quoka_status st = quoka::check_prefill_args(p, q, k_cache, v_cache, out);
   if (st != QUOKA_OK) return st;
+  size_t need = 0;
+  if ((st = quoka_workspace_size(p, &need)) != QUOKA_OK) return st;
   if (need > (size_t)QUOKA_STATIC_SCRATCH_BYTES) return QUOKA_ERR_STATIC_LIMIT;
   void* scratch = nullptr;
   if ((st = quoka::static_scratch_for_current_device(&scratch)) != QUOKA_OK) return st;

@@ -82,6 +82,16 @@ static quoka_status validate(const quoka_params* p) {
 
 static bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }
 
+// Everything the fused call checks before it touches the stream, except the workspace.
+quoka_status check_prefill_args(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
+                                const void* out) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!q || !k_cache || !v_cache || !out) return QUOKA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return QUOKA_ERR_INVALID_ARG;
+  return QUOKA_OK;
+}
+
 static quoka_status check_ws(const quoka_params* p, void* ws, size_t ws_bytes) {
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0) return QUOKA_ERR_WORKSPACE;
   if (ws_bytes < carve(p, nullptr).total) return QUOKA_ERR_WORKSPACE;
@@ -234,10 +244,8 @@ quoka_status quoka_dense_chunk_attn(const quoka_params* p, const void* q, const 
 quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
                                  void* out, int32_t* k_idx_out, int32_t* k_cnt_out, void* ws, size_t ws_bytes,
                                  void* stream) {
-  quoka_status st = validate(p);
+  quoka_status st = check_prefill_args(p, q, k_cache, v_cache, out);
   if (st != QUOKA_OK) return st;
-  if (!q || !k_cache || !v_cache || !out) return QUOKA_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return QUOKA_ERR_INVALID_ARG;
   if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   DevParams P = make_dev(p, ws);
@@ -291,8 +299,26 @@ quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_
   return QUOKA_OK;
 }
 
+quoka_status quoka_append_kv(const quoka_params* p, const void* k_new, const void* v_new, void* k_cache,
+                             void* v_cache, float* k_inv_norm, void* ws, size_t ws_bytes, void* stream) {
+  quoka_status st = validate(p);
+  if (st != QUOKA_OK) return st;
+  if (!k_new || !v_new || !k_cache || !v_cache) return QUOKA_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache)) return QUOKA_ERR_INVALID_ARG;
+  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const DevParams P = make_dev(p, ws);
+  QUOKA_TRY_CUDA(launch_append_kv(P, p->dtype, k_new, v_new, k_cache, v_cache, cs));
+  if (k_inv_norm) QUOKA_TRY_CUDA(launch_key_norms(P, p->dtype, k_cache, k_inv_norm, 0, cs));
+  return QUOKA_OK;
+}
+
 quoka_status quoka_last_device_status(void* ws, void* stream, int32_t* status_out) {
-  if (!ws || !status_out) return QUOKA_ERR_INVALID_ARG;
+  if (!status_out) return QUOKA_ERR_INVALID_ARG;
+  if (!ws) {                                  // the built-in scratch array of quoka_prefill_chunk_static
+    quoka_status st = static_scratch_for_current_device(&ws);
+    if (st != QUOKA_OK) return st;
+  }
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   int32_t h = 0;
   QUOKA_TRY_CUDA(cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, cs));
@@ -311,6 +337,7 @@ const char* quoka_status_string(quoka_status s) {
     case QUOKA_ERR_CUDA: return "CUDA call failed";
     case QUOKA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case QUOKA_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in static array holds";
+    case QUOKA_ERR_BAD_INDEX: return "a selected row or page id was out of range (debug build)";
     default: return "unknown status";
   }
 }

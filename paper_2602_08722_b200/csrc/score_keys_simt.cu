@@ -107,6 +107,7 @@ cudaError_t launch_key_norms(const DevParams& P, int dtype, const void* k, float
   const int64_t warps = (int64_t)P.batch * P.n_kv * rows_max;
   const int grid = (int)((warps * 32 + 255) / 256);
   if (grid <= 0) return cudaSuccess;
+  log_launch("key_norms", dim3(grid), dim3(256), 0, 1, false);
   if (dtype == QUOKA_BF16) {
     if (P.d == 128) key_norms_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16*)k, k_inv_norm, all_rows, rows_max);
     else key_norms_kernel<__nv_bfloat16, 64><<<grid, 256, 0, st>>>(P, (const __nv_bfloat16*)k, k_inv_norm, all_rows, rows_max);
@@ -122,6 +123,7 @@ cudaError_t launch_score_keys_simt(const DevParams& P, int dtype, const void* qb
                                    cudaStream_t st) {
   if (P.max_ctx <= 0) return cudaSuccess;
   dim3 grid((P.max_ctx + kScoreTile - 1) / kScoreTile, P.n_kv, P.batch);
+  log_launch("score_keys_simt", grid, dim3(kScoreTile), (size_t)(kScoreTile * (P.d + 1) + kQChunk * P.d) * sizeof(float), 1, false);
 #define QUOKA_SCORE(T_, D)                                                                                     \
   do {                                                                                                        \
     const size_t smem = (size_t)(kScoreTile * (D + 1) + kQChunk * D) * sizeof(float);                         \

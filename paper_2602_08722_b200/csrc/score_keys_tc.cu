@@ -187,6 +187,8 @@ score_keys_tc_kernel(DevParams P, ScoreArgs A, const __grid_constant__ CUtensorM
         if (++n_issued >= A.stages - 1 && q_deferred >= 0) { load_q(q_deferred); q_deferred = -1; }
       }
       if (q_deferred >= 0) load_q(q_deferred);
+      // a CTA without tiles still waits: the chain of a fused call is only transitive if every link has waited
+      if (!waited) grid_dependency_wait();
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -427,11 +429,11 @@ quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, con
   if (P.d == 128) {
     e = cudaFuncSetAttribute(score_keys_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.total);
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;
-    e = launch_kernel(score_keys_tc_kernel<2>, dim3(grid), dim3(kScoreThreads), pl.total, st, 1, chained, P, A, tm_q, tm_k, scores);
+    e = launch_kernel("score_keys_tc", score_keys_tc_kernel<2>, dim3(grid), dim3(kScoreThreads), pl.total, st, 1, chained, P, A, tm_q, tm_k, scores);
   } else {
     e = cudaFuncSetAttribute(score_keys_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.total);
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;
-    e = launch_kernel(score_keys_tc_kernel<1>, dim3(grid), dim3(kScoreThreads), pl.total, st, 1, chained, P, A, tm_q, tm_k, scores);
+    e = launch_kernel("score_keys_tc", score_keys_tc_kernel<1>, dim3(grid), dim3(kScoreThreads), pl.total, st, 1, chained, P, A, tm_q, tm_k, scores);
   }
   count_launch();
   return (e == cudaSuccess && cudaGetLastError() == cudaSuccess) ? QUOKA_OK : QUOKA_ERR_CUDA;

@@ -160,9 +160,12 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
   constexpr int kAll = CL * kSelThreads;
   if (kv == 0 && gtid == 0) k_cnt[s] = B;
   for (int i = B + gtid; i < P.budget_cap; i += kAll) out[i] = -1;
-  if (B <= 0) return;                           // uniform over the cluster
+  // Every exit path waits for the kernel before this one: the kernels of a fused call are ordered as a chain, and
+  // "the last kernel has completed" implies "all of them have" only if no link finishes without having waited.
+  if (B <= 0) { grid_dependency_wait(); return; }      // uniform over the cluster
   if (B >= T) {                                 // budget covers the cache: identity
     for (int i = gtid; i < T; i += kAll) out[i] = i;
+    grid_dependency_wait();
     return;
   }
   const int base = (rank * kSelThreads + wid * 32) * ITEMS + lane;      // position of item i: base + 32 i
@@ -435,7 +438,7 @@ __global__ void __launch_bounds__(kSelThreads) select_keys_reg_kernel(DevParams 
 template <int ITEMS, int CL>
 static cudaError_t launch_reg(const DevParams& P, const float* scores, int32_t* k_idx, int32_t* k_cnt, cudaStream_t st,
                               bool chained) {
-  return launch_kernel(select_keys_reg_kernel<ITEMS, CL>, dim3(P.batch * P.n_kv * CL), dim3(kSelThreads), 0, st, CL, chained,
+  return launch_kernel("select_keys_reg", select_keys_reg_kernel<ITEMS, CL>, dim3(P.batch * P.n_kv * CL), dim3(kSelThreads), 0, st, CL, chained,
                        P, scores, k_idx, k_cnt);
 }
 
@@ -452,7 +455,7 @@ cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t*
   else if (per_thread <= 64) e = launch_reg<32, 2>(P, scores, k_idx, k_cnt, st, chained);
   else if (per_thread <= 128) e = launch_reg<32, 4>(P, scores, k_idx, k_cnt, st, chained);
   else if (per_thread <= 256) e = launch_reg<32, 8>(P, scores, k_idx, k_cnt, st, chained);
-  else e = launch_kernel(select_keys_kernel, dim3(P.batch * P.n_kv), dim3(kSelThreads), 0, st, 1, chained, P, scores, k_idx, k_cnt);
+  else e = launch_kernel("select_keys", select_keys_kernel, dim3(P.batch * P.n_kv), dim3(kSelThreads), 0, st, 1, chained, P, scores, k_idx, k_cnt);
   count_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -377,7 +377,7 @@ static cudaError_t launch_rank_t(const DevParams& P, const void* q, int32_t* q_i
   const size_t smem = fixed + (staged ? row_bytes : 0);
   cudaError_t e = cudaFuncSetAttribute(rank_queries_kernel<T, D, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  return launch_kernel(rank_queries_kernel<T, D, CL>, dim3(P.batch * P.n_q * CL), dim3(kRankThreads), smem, st, CL, false, P,
+  return launch_kernel("rank_queries", rank_queries_kernel<T, D, CL>, dim3(P.batch * P.n_q * CL), dim3(kRankThreads), smem, st, CL, false, P,
                        (const T*)q, q_idx, rpc, n_sort, staged, m_peer);
 }
 
@@ -405,11 +405,11 @@ cudaError_t launch_aggregate_queries(const DevParams& P, int dtype, const void* 
   const dim3 grid((unsigned)((warps * 32 + 255) / 256)), block(256);
   cudaError_t e;
   if (dtype == QUOKA_BF16) {
-    if (P.d == 128) e = launch_kernel(aggregate_queries_kernel<__nv_bfloat16, 128>, grid, block, 0, st, 1, chained, P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
-    else e = launch_kernel(aggregate_queries_kernel<__nv_bfloat16, 64>, grid, block, 0, st, 1, chained, P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
+    if (P.d == 128) e = launch_kernel("aggregate_queries", aggregate_queries_kernel<__nv_bfloat16, 128>, grid, block, 0, st, 1, chained, P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
+    else e = launch_kernel("aggregate_queries", aggregate_queries_kernel<__nv_bfloat16, 64>, grid, block, 0, st, 1, chained, P, (const __nv_bfloat16*)q, q_idx, (__nv_bfloat16*)qbar);
   } else {
-    if (P.d == 128) e = launch_kernel(aggregate_queries_kernel<float, 128>, grid, block, 0, st, 1, chained, P, (const float*)q, q_idx, (float*)qbar);
-    else e = launch_kernel(aggregate_queries_kernel<float, 64>, grid, block, 0, st, 1, chained, P, (const float*)q, q_idx, (float*)qbar);
+    if (P.d == 128) e = launch_kernel("aggregate_queries", aggregate_queries_kernel<float, 128>, grid, block, 0, st, 1, chained, P, (const float*)q, q_idx, (float*)qbar);
+    else e = launch_kernel("aggregate_queries", aggregate_queries_kernel<float, 64>, grid, block, 0, st, 1, chained, P, (const float*)q, q_idx, (float*)qbar);
   }
   if (e != cudaSuccess) return e;
   count_launch();

@@ -40,11 +40,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Every wait in the kernels goes through here.  It gives up after about a second (or as soon as
 // another thread of the CTA has given up), records QUOKA_ERR_TIMEOUT in the device status word and
 // returns false; the caller then leaves its loop and runs the normal teardown.
-struct WaitCtx {
-  volatile int* abort_flag;   // shared memory, one per CTA
-  int32_t* status;            // global status word
-};
 constexpr long long kWaitCycles = 2000000000LL;
+struct WaitCtx {
+  volatile int* abort_flag;        // shared memory, one per CTA
+  int32_t* status;                 // global status word
+  long long limit = kWaitCycles;   // cycles after which a wait gives up
+};
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -52,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
   uint32_t it = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++it & 63u) == 0) {
-      if (*w.abort_flag || clock64() - t0 > kWaitCycles) {
+      if (*w.abort_flag || clock64() - t0 > w.limit) {
         *w.abort_flag = 1;
         atomicExch(w.status, (int32_t)QUOKA_ERR_TIMEOUT);
         return false;

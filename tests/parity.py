@@ -5,7 +5,8 @@ oracle within that stage's tie rule, then the CUDA output itself (not the
 oracle's) is fed to the oracle's next stage.  Index work is bit-exact up to ties:
 a rank or a key may differ from the oracle's only where the oracle's own score
 gap is below 1e-4 relative.  Attention outputs on identical indices: bf16 within
-2e-2 max-abs and 2e-3 mean-abs; f32 within 2e-4 / 2e-5.
+2e-2 max-abs (outputs below 4 in magnitude; see attention_bound for larger ones)
+and 2e-3 mean-abs; f32 within 2e-4 / 2e-5.
 """
 from __future__ import annotations
 
@@ -84,12 +85,35 @@ def check_key_selection(k_idx_gpu: np.ndarray, scores_oracle: np.ndarray, B: int
     return diffs
 
 
+def attention_bound(out_oracle: np.ndarray, dtype: str) -> np.ndarray:
+    """Element-wise bound on |out_gpu - out_oracle|.
+
+    f32: 2e-4 everywhere.  bf16: the stated 2e-2 max-abs wherever |o| < 4.  An output of magnitude 4 or more is
+    STORED in bf16 with a spacing of 2^-5 or more, so rounding the exact result alone may cost half a spacing
+    (0.0156 for 4 <= |o| < 8) and leaves the arithmetic under 0.0044 of the 2e-2; there the bound is half a bf16
+    spacing of |o| plus 2^-8 |o| (bf16 softmax weights in the PV product: 2^-9 relative each, on a row dominated by
+    few keys they do not average out, and the row sum is taken before the rounding)."""
+    mx, _ = ATTN_TOL[dtype]
+    a = np.abs(out_oracle)
+    bound = np.full(a.shape, mx)
+    if dtype == "bf16":
+        big = a >= 4.0
+        spacing = 2.0 ** (np.floor(np.log2(np.maximum(a, 4.0))) - 7)
+        bound = np.where(big, spacing / 2 + a * 2.0 ** -8, bound)
+    return bound
+
+
 def check_attention(out_gpu: np.ndarray, out_oracle: np.ndarray, dtype: str):
+    """Returns the number of elements judged by the large-output bound (|o| >= 4, bf16 only)."""
     diff = np.abs(out_gpu - out_oracle)
-    mx, mean = ATTN_TOL[dtype]
+    _, mean = ATTN_TOL[dtype]
     assert np.isfinite(out_gpu).all()
-    assert diff.max() <= mx, f"attention max abs diff {diff.max()} > {mx}"
+    bound = attention_bound(out_oracle, dtype)
+    worst = np.unravel_index(np.argmax(diff - bound), diff.shape)
+    assert (diff <= bound).all(), (f"attention abs diff {diff[worst]} > {bound[worst]} at {worst} "
+                                   f"(oracle value {out_oracle[worst]})")
     assert diff.mean() <= mean, f"attention mean abs diff {diff.mean()} > {mean}"
+    return int((np.abs(out_oracle) >= 4.0).sum()) if dtype == "bf16" else 0
 
 
 class GpuProblem:
@@ -153,9 +177,24 @@ class GpuProblem:
         return q, k, v, T
 
 
+def stratified_rows(n_q: int, C: int, n_random: int, seed: int):
+    """(heads, rows) for a sampled attention check: for EVERY head the rows at the edges of the kernels' 128-row
+    tiles (0, 127, 128, 255, 256, the last row, and the rows around the middle tile edge), then n_random uniformly
+    drawn pairs."""
+    mid = (C // 2) // 128 * 128
+    edges = sorted({r for r in (0, 127, 128, 255, 256, mid - 1, mid, C - 129, C - 128, C - 1) if 0 <= r < C})
+    heads = np.repeat(np.arange(n_q), len(edges))
+    rows = np.tile(np.array(edges, dtype=np.int64), n_q)
+    r = np.random.default_rng(seed)
+    heads = np.concatenate([heads, r.integers(0, n_q, n_random)])
+    rows = np.concatenate([rows, r.integers(0, C, n_random)])
+    return heads, rows
+
+
 def check_chain(gp: GpuProblem, attn_rows=None, seed=0):
-    """Validate every stage of a staged run against the oracle.  attn_rows: number of
-    sampled (head, row) pairs per sequence for the attention check (None = all rows)."""
+    """Validate every stage of a staged run against the oracle.  attn_rows: number of randomly
+    sampled (head, row) pairs per sequence for the attention check, on top of the tile-edge rows
+    of every head (None = all rows)."""
     stats = dict(rank_swaps=0, key_diffs=0)
     for s in range(gp.b):
         q, k, v, T = gp.oracle_inputs(s)
@@ -195,13 +234,10 @@ def check_chain(gp: GpuProblem, attn_rows=None, seed=0):
         out_g = f64(gp.out[s])
         if attn_rows is None:
             out_o, lse_o = O.sparse_attention(q, k, v, T, idx_list)
-            check_attention(out_g, out_o, gp.dtype)
+            stats["big_outputs"] = stats.get("big_outputs", 0) + check_attention(out_g, out_o, gp.dtype)
             assert np.abs(f64(gp.lse[s]) - lse_o).max() <= 2e-3
         else:
-            r = np.random.default_rng(seed + s)
-            heads = r.integers(0, gp.n_q, attn_rows)
-            rows = r.integers(0, gp.C, attn_rows)
-            rows[0], rows[1] = 0, gp.C - 1
+            heads, rows = stratified_rows(gp.n_q, gp.C, attn_rows, seed + s)
             out_o = O.sparse_attention_rows(q, k, v, T, idx_list, heads, rows)
-            check_attention(out_g[heads, rows], out_o, gp.dtype)
+            stats["big_outputs"] = stats.get("big_outputs", 0) + check_attention(out_g[heads, rows], out_o, gp.dtype)
     return stats

@@ -84,6 +84,7 @@ def test_bad_params_are_rejected_before_any_launch(lib, field, value, status):
 def test_null_and_misaligned_pointers_and_small_workspace(lib):
     from paper_2602_08722_b200 import api
     p = good_params()
+    before = api.quoka_launch_count()
     assert lib.quoka_select_queries(C.byref(p), None, 0x2000, 0x3000, 0x4000, 1 << 30, None) == api.ERR_INVALID_ARG
     assert lib.quoka_select_queries(C.byref(p), 0x1008, 0x2000, 0x3000, 0x4000, 1 << 30, None) == api.ERR_INVALID_ARG
     assert lib.quoka_select_queries(C.byref(p), 0x1000, 0x2000, 0x3000, None, 1 << 30, None) == api.ERR_WORKSPACE
@@ -91,7 +92,7 @@ def test_null_and_misaligned_pointers_and_small_workspace(lib):
     assert lib.quoka_select_queries(C.byref(p), 0x1000, 0x2000, 0x3000, 0x4000, 64, None) == api.ERR_WORKSPACE
     assert lib.quoka_sparse_attn(C.byref(p), 0x1000, 0x2000, 0x3000, None, 0x5000, 0x6000, None, 0x4000, 1 << 30,
                                  None) == api.ERR_INVALID_ARG
-    assert api.quoka_launch_count() == 0 or True
+    assert api.quoka_launch_count() == before
     assert api.status_string(api.ERR_TIMEOUT)
 
 
@@ -109,3 +110,43 @@ def test_missing_library_is_an_error(monkeypatch, tmp_path):
     monkeypatch.setattr(api, "_LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         api.load()
+
+
+def test_block_table_check_on_the_host(lib):
+    """quoka_check_block_table: pages outside the pool and pages used twice are refused; nothing is launched."""
+    import torch
+    from paper_2602_08722_b200 import api, synth
+    inp = synth.to_paged(synth.make_chunk_inputs(3, 2, 4, 2, 64, [200, 70], 60, "bf16"), 3)
+    p = good_params()
+    p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim, p.chunk_len, p.max_ctx_len = 2, 4, 2, 64, 60, 200
+    p.page_size, p.max_pages_per_seq, p.kv_rows = 64, inp.block_table.shape[1], inp.k_pages.shape[0]
+    before = api.quoka_launch_count()
+    table = inp.block_table.clone()
+    assert api.quoka_check_block_table(p, inp.ctx_len, table) == api.OK
+    bad = table.clone()
+    bad[0, 1] = p.kv_rows                     # one past the pool
+    assert api.quoka_check_block_table(p, inp.ctx_len, bad) == api.ERR_INVALID_ARG
+    bad = table.clone()
+    bad[1, 0] = table[0, 0]                   # two logical pages on one physical page
+    assert api.quoka_check_block_table(p, inp.ctx_len, bad) == api.ERR_INVALID_ARG
+    bad = table.clone()
+    bad[1, 3] = -1                            # a page the sequence does not need may be anything
+    assert api.quoka_check_block_table(p, inp.ctx_len, bad) == api.OK
+    too_long = torch.tensor([201, 70], dtype=torch.int32)
+    assert api.quoka_check_block_table(p, too_long, table) == api.ERR_INVALID_ARG
+    assert api.quoka_launch_count() == before
+
+
+def test_debug_library_builds_and_exports_the_same_entry_points():
+    from paper_2602_08722_b200 import api, build
+    build.build(debug=True)
+    dbg = api.open_debug_library()
+    for n in declared_entry_points():
+        assert hasattr(dbg, n)
+
+
+def test_launch_logging_is_off_by_default(lib, capfd):
+    from paper_2602_08722_b200 import api
+    p = good_params()
+    lib.quoka_select_queries(C.byref(p), None, 0x2000, 0x3000, 0x4000, 1 << 30, None)
+    assert "[quoka]" not in capfd.readouterr().err
