@@ -2,6 +2,8 @@
 """Benchmark of the QuoKA per-chunk prefill path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+    python bench.py --grid      timing sweep at 32K context (budget x chunk x head_dim x GQA x retained queries)
+    python bench.py --sweep     Algorithm 2 over a whole prompt (append, select, attend per chunk)
 
 One "step" = one pass of the whole hot path (query sub-selection, key scoring, top-B
 selection, sparse attention: the fused quoka_prefill_chunk call) over one prefill chunk
@@ -9,8 +11,12 @@ of synthetic input.  The metric is microseconds per prefill chunk (lower is bett
 With N > 1 (torchrun, one rank per GPU) every rank processes its own independent chunk:
 weak scaling, no data-path collective.  Rank 0 prints ONE JSON line.
 
+The default line also carries, under "configs", the same measurements for the other named
+workloads (128K long context, paged serving mix, tiny), taken after the timed region.
+
 --impl reference times the CPU oracle (the only other program in this repository that
-computes the path) on the host cores, on a bounded sample of the same workload.
+computes the path) on the host cores: in full where one pass costs a few seconds, on a
+bounded sample of the same workload otherwise.
 """
 from __future__ import annotations
 
@@ -30,9 +36,16 @@ import torch  # noqa: E402
 
 METRIC = "us_per_prefill_chunk"
 UNIT = "us"
-# DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu capture of that workload
-# (profiles/kernels_full_<workload>.md); None where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {("llama8b_32k", "sparse_attn"): 42.5e6}
+# DRAM bytes (read + write) per launch of a kernel, taken from the committed ncu captures: a small table beside
+# the summaries, keyed "<workload>/<kernel>"; a kernel that changed since its capture has no entry.
+def ncu_traffic(workload, kernel):
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        return json.load(open(path)).get(f"{workload}/{kernel}", {}).get("dram_bytes_per_launch")
+    except (OSError, ValueError):
+        return None
+
+
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -213,11 +226,14 @@ def time_loop(fn, steps, warmup, flush):
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(w, ctx_lens, seed, budget_s=15.0):
-    """Times the oracle, as it stands, on sequence 0 of the workload: selection in full,
-    attention in full for the first `ng` KV groups (all rows of their G query heads), with ng
-    chosen so the run costs about `budget_s` seconds; the attention time is scaled by
-    n_KV / ng and the total by the batch's cached length.  Returns (us per chunk, sample, seconds)."""
+FULL_ORACLE_FLOPS = 2.5e11      # one pass of the oracle in full below this many attention flops (about 8 s of host time)
+
+
+def oracle_sample(w, ctx_lens, seed, budget_s=15.0, allow_full=True):
+    """Times the oracle, as it stands, on sequence 0 of the workload: selection in full, attention in full for
+    the first `ng` KV groups (all rows of their G query heads).  ng = all groups when the whole pass is cheap
+    (then nothing is extrapolated), else chosen so the run costs about `budget_s` seconds, the attention time
+    scaled by n_KV / ng; a batch is scaled by its cached length.  Returns (us per chunk, sample, seconds)."""
     import numpy as np
     from oracle import quoka_oracle as O
     from paper_2602_08722_b200 import synth
@@ -236,15 +252,31 @@ def oracle_sample(w, ctx_lens, seed, budget_s=15.0):
     k_idx = O.select_keys(scores, B)
     t_sel = time.perf_counter() - t0
     flops_group = 4.0 * G * C * w["d"] * (B + C / 2)
-    ng = int(max(1, min(n_kv, round(max(budget_s - t_sel, 0.5) * 13e9 / flops_group))))
+    if allow_full and flops_group * n_kv <= FULL_ORACLE_FLOPS:
+        ng = n_kv
+    else:
+        ng = int(max(1, min(n_kv, round(max(budget_s - t_sel, 0.5) * 13e9 / flops_group))))
     t0 = time.perf_counter()
-    O.sparse_attention(q[: ng * G], k[:ng], v[:ng], T, k_idx[:ng])
-    t_att = time.perf_counter() - t0
+    if ng * flops_group > 4 * budget_s * 13e9:
+        # even one KV group is too much (128K): a stated subsample of the rows of its G heads, one by one
+        n_rows = 512
+        r = np.random.default_rng(seed)
+        heads, rows = r.integers(0, G, n_rows), r.integers(0, C, n_rows)
+        O.sparse_attention_rows(q[:G], k[:1], v[:1], T, k_idx[:1], heads, rows)
+        t_att = (time.perf_counter() - t0) * (G * C / n_rows)
+        spent = time.perf_counter() - t0
+        what = f"attention on {n_rows} sampled rows of KV group 0 (extrapolated x{G * C / n_rows:.0f} to the group, x{n_kv} to all groups)"
+        ng = 1
+    else:
+        O.sparse_attention(q[: ng * G], k[:ng], v[:ng], T, k_idx[:ng])
+        t_att = spent = time.perf_counter() - t0
+        what = (f"attention in full for all {n_kv} KV groups (nothing extrapolated)" if ng == n_kv else
+                f"attention in full for {ng} of {n_kv} KV groups (extrapolated x{n_kv}/{ng})")
     per_chunk_s = t_sel + t_att * n_kv / ng
     scale_batch = sum(ctx_lens) / float(T) if (len(ctx_lens) > 1 and T > 0) else float(len(ctx_lens))
-    sample = (f"sequence 0 of {len(ctx_lens)}: selection in full, attention in full for {ng} of {n_kv} KV groups "
-              f"(scaled by {n_kv}/{ng})" + (f", batch scaled by cached length x{scale_batch:.2f}" if len(ctx_lens) > 1 else ""))
-    return per_chunk_s * 1e6 * scale_batch, sample, t_sel + t_att
+    sample = (f"sequence 0 of {len(ctx_lens)}: selection in full, " + what +
+              (f", batch extrapolated by cached length x{scale_batch:.2f}" if len(ctx_lens) > 1 else ""))
+    return per_chunk_s * 1e6 * scale_batch, sample, t_sel + spent
 
 
 def host_threads():
@@ -256,31 +288,182 @@ def host_threads():
         return os.cpu_count() or 1
 
 
-# ----------------------------------------------------------------------------- whole-prompt sweep
-def sweep(args, w, q, k, v, out, ctx, dev, rank):
-    """Algorithm 2 over a whole prompt of T + C tokens: chunk i sees T_i = i*C cached rows (the synthetic cache rows
-    stand in for the keys earlier chunks would have appended).  Budget = 12 % of the cached length per chunk."""
-    from paper_2602_08722_b200 import api
-    T, C = w["T"], w["C"]
-    lens = list(range(0, T + 1, C))
-    frac = 0.12
-    ps = [api.make_params(q, k, out, ctx, n_retain=w["n_retain"], kv_budget=0, budget_frac=frac, max_ctx_len=t)
-          for t in lens]
-    for p_i in ps:
-        p_i.kv_rows = k.shape[2]
-    ws = api.alloc_workspace(ps[-1])
-    len_dev = [torch.tensor([t], dtype=torch.int32, device=dev) for t in lens]
+# ----------------------------------------------------------------------------- one workload on the device
+class Problem:
+    """Device buffers and parameters of one workload (inputs drawn on the host from the seeded generator, or, for
+    the timing-only grid, drawn on the device)."""
 
-    def chunk(i, dense):
-        ctx.copy_(len_dev[i])                                   # device-to-device on the stream: graph-safe
-        if dense:
-            api.quoka_dense_chunk_attn(ps[i], q, k, v, out, None, ws)
+    def __init__(self, w, seed, ctx_lens, dev, impl=0, cached_norms=False, on_device=False):
+        from paper_2602_08722_b200 import api, synth
+        self.w, self.ctx_lens, self.dev = w, ctx_lens, dev
+        paged = bool(w.get("paged"))
+        self.paged = paged
+        if on_device:
+            g = torch.Generator(device=dev).manual_seed(seed)
+            b, n_q, n_kv, d, C = w["batch"], w["n_q"], w["n_kv"], w["d"], w["C"]
+            rows = max(ctx_lens) + C
+            mu = torch.randn(b, n_q, 1, d, device=dev, generator=g)
+            self.q = (mu + 0.7 * torch.randn(b, n_q, C, d, device=dev, generator=g)).to(torch.bfloat16)
+            k = torch.randn(b, n_kv, rows, d, device=dev, generator=g)
+            k = torch.where(torch.rand(b, n_kv, rows, 1, device=dev, generator=g) < 0.05, k * 3.0, k)
+            self.k = k.to(torch.bfloat16)
+            self.v = torch.randn(b, n_kv, rows, d, device=dev, generator=g).to(torch.bfloat16)
+            self.bt = None
+            self.ctx = torch.tensor(ctx_lens, dtype=torch.int32, device=dev)
+            self.inp = None
         else:
-            api.quoka_prefill_chunk(ps[i], q, k, v, out, None, None, ws)
+            inp = synth.make_chunk_inputs(seed, w["batch"], w["n_q"], w["n_kv"], w["d"], ctx_lens, w["C"], w["dtype"])
+            if paged:
+                inp = synth.to_paged(inp, seed)
+            self.inp = inp
+            self.q = inp.q.to(dev)
+            self.k = (inp.k_pages if paged else inp.k).to(dev)
+            self.v = (inp.v_pages if paged else inp.v).to(dev)
+            self.bt = inp.block_table.to(dev) if paged else None
+            self.ctx = inp.ctx_len.to(dev)
+        self.out = torch.zeros_like(self.q)
+        self.p = api.make_params(self.q, self.k, self.out, self.ctx, n_retain=w["n_retain"],
+                                 kv_budget=w.get("kv_budget", 0), budget_frac=w.get("budget_frac", 0.0),
+                                 max_ctx_len=max(ctx_lens), block_table=self.bt, impl=impl)
+        self.ws = api.alloc_workspace(self.p)
+        self.k_inv_norm = None
+        if cached_norms:
+            self.k_inv_norm = torch.zeros(tuple(self.k.shape[:3]), dtype=torch.float32, device=dev)
+            api.quoka_update_key_norms(self.p, self.k, self.k_inv_norm, True, self.ws)
+            self.p.k_inv_norm = self.k_inv_norm.data_ptr()
+        cap = api.quoka_kv_budget_cap(self.p)
+        b, n_q, C, d = self.q.shape
+        n_kv = self.k.shape[1]
+        N = min(w["n_retain"], C)
+        self.q_idx = torch.zeros((b, n_q, N), dtype=torch.int32, device=dev)
+        self.qbar = torch.zeros((b, n_kv, N, d), dtype=self.q.dtype, device=dev)
+        self.scores = torch.zeros((b, n_kv, max(max(ctx_lens), 1)), dtype=torch.float32, device=dev)
+        self.k_idx = torch.zeros((b, n_kv, cap), dtype=torch.int32, device=dev)
+        self.k_cnt = torch.zeros((b,), dtype=torch.int32, device=dev)
+
+    def step(self):
+        from paper_2602_08722_b200 import api
+        api.quoka_prefill_chunk(self.p, self.q, self.k, self.v, self.out, None, None, self.ws)
+
+    def dense(self):
+        from paper_2602_08722_b200 import api
+        api.quoka_dense_chunk_attn(self.p, self.q, self.k, self.v, self.out, None, self.ws)
+
+    def stages(self):
+        from paper_2602_08722_b200 import api
+        return {
+            "select_queries": lambda: api.quoka_select_queries(self.p, self.q, self.q_idx, self.qbar, self.ws),
+            "score_keys": lambda: api.quoka_score_keys(self.p, self.qbar, self.k, self.scores, self.ws),
+            "select_keys": lambda: api.quoka_select_keys(self.p, self.scores, self.k_idx, self.k_cnt, self.ws),
+            "sparse_attn": lambda: api.quoka_sparse_attn(self.p, self.q, self.k, self.v, self.k_idx, self.k_cnt,
+                                                         self.out, None, self.ws),
+        }
+
+
+def per_kernel(prob, ksteps, flush, pk, workload):
+    """Per-kernel timings: the staged entry points run back to back on the stream, exactly as the fused call
+    issues them, with a CUDA event between stages (a kernel timed alone after an idle stream carries ~10 us of
+    launch latency, which hides the small kernels); L2 is flushed before each sequence.  Then the dense kernel."""
+    w = prob.w
+    stages = prob.stages()
+    work = sum_work(w, prob.ctx_lens)
+    samples = {name: [] for name in stages}
+    for it in range(ksteps + 3):
+        flush()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)]
+        evs[0].record()
+        for i, fn in enumerate(stages.values()):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            for i, name in enumerate(stages):
+                samples[name].append(evs[i].elapsed_time(evs[i + 1]) * 1e3)
+    kernels = {}
+    for name in stages:
+        ts = samples[name]
+        us = statistics.mean(ts)
+        kernels[name] = {"us": round(us, 2), "min_us": round(min(ts), 2),
+                         "gbs": round(work[name]["bytes"] / us / 1e3, 1),
+                         "tflops": round(work[name]["flops"] / us / 1e6, 2)}
+    dense_steps = 3 if work["dense_attn"]["flops"] > 2e12 else ksteps
+    ts = time_loop(prob.dense, dense_steps, 1, flush)
+    us = statistics.mean(ts)
+    kernels["dense_attn"] = {"us": round(us, 2), "min_us": round(min(ts), 2),
+                             "gbs": round(work["dense_attn"]["bytes"] / us / 1e3, 1),
+                             "tflops": round(work["dense_attn"]["flops"] / us / 1e6, 2)}
+    for name, bound in (("select_queries", "hbm"), ("score_keys", "hbm"), ("select_keys", "hbm"),
+                        ("sparse_attn", "tensor"), ("dense_attn", "tensor")):
+        kk = kernels[name]
+        kk["bound"] = bound
+        kk["frac"] = round(kk["gbs"] / pk["hbm_gbs"], 4) if bound == "hbm" else round(kk["tflops"] / pk["bf16_tflops"], 4)
+    # scoring is tensor-bound once N exceeds the ridge point (flop per byte of K)
+    if work["score_keys"]["flops"] / (pk["bf16_tflops"] * 1e12) > work["score_keys"]["bytes"] / (pk["hbm_gbs"] * 1e9):
+        kernels["score_keys"]["bound"] = "tensor"
+        kernels["score_keys"]["frac"] = round(kernels["score_keys"]["tflops"] / pk["bf16_tflops"], 4)
+    for name in kernels:
+        kernels[name]["ncu_dram_bytes"] = ncu_traffic(workload, name)
+    return kernels, round(sum(kernels[n]["us"] for n in stages), 2)
+
+
+def side_config(name, seed, dev, flush, pk, steps, cpu_leg):
+    """The measurements of the default line for another named workload: fused us per chunk, every kernel, the
+    dense kernel, the speed-up, the oracle on the host cores."""
+    from paper_2602_08722_b200 import api, synth
+    w = dict(synth.WORKLOADS[name])
+    _, ctx_lens = rank_workload(w, seed, 0)
+    prob = Problem(w, seed, ctx_lens, dev)
+    ts = time_loop(prob.step, steps, 3, flush)
+    fused = statistics.mean(ts)
+    kernels, staged_sum = per_kernel(prob, max(3, min(steps, 10)), flush, pk, name)
+    res = {"us_per_prefill_chunk": round(fused, 2), "min_us": round(min(ts), 2), "steps": steps,
+           "ctx_len": w["T"] if w["T"] is not None else ctx_lens, "chunk_len": w["C"], "n_retain": w["n_retain"],
+           "kv_budget": w.get("kv_budget", 0), "budget_frac": w.get("budget_frac", 0.0), "batch": w["batch"],
+           "paged": bool(w.get("paged")), "dtype": w["dtype"], "kernels": kernels, "staged_sum_us": staged_sum,
+           "dense_us": kernels["dense_attn"]["us"],
+           "speedup_vs_dense_chunk_attn": round(kernels["dense_attn"]["us"] / fused, 3),
+           "device_status": api.quoka_last_device_status(prob.ws)}
+    del prob
+    torch.cuda.empty_cache()
+    if cpu_leg:
+        us_cpu, sample, secs = oracle_sample(w, ctx_lens, seed, budget_s=10.0)
+        res["cpu_baseline"] = {"value": round(us_cpu, 1), "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                               "sample": sample, "cpu_seconds_spent": round(secs, 2)}
+    return res
+
+
+# ----------------------------------------------------------------------------- whole-prompt sweep (Algorithm 2)
+def sweep(args, w, dev, rank):
+    """Algorithm 2 over a whole prompt of T + C tokens with a cache that really grows: the device cache starts
+    empty; chunk i appends its K_i, V_i (quoka_append_kv, from a device copy of the prompt's keys and values),
+    runs the loop body at cached length i*C, and the cached length advances on the device.  Timed as eager calls,
+    as ONE CUDA graph of the whole prompt, and with the dense chunk kernel in place of QuoKA.  Budget = 12 % of
+    the cached length per chunk."""
+    from paper_2602_08722_b200 import api
+    T, C = w["T"], (args.chunk if args.chunk else w["C"])
+    w = dict(w, C=C, kv_budget=0, budget_frac=0.12)
+    lens = list(range(0, T + 1, C))
+    prob = Problem(w, args.seed, [T], dev, on_device=True)
+    q, k, v, out, ctx = prob.q, prob.k, prob.v, prob.out, prob.ctx
+    k_all, v_all = k.clone(), v.clone()                       # the prompt's K, V; rows [iC, (i+1)C) = chunk i
+    ps = []
+    for t in lens:
+        p_i = api.make_params(q, k, out, ctx, n_retain=w["n_retain"], kv_budget=0, budget_frac=0.12, max_ctx_len=t)
+        p_i.kv_rows = k.shape[2]
+        ps.append(p_i)
+    ws = api.alloc_workspace(ps[-1])
+    chunks_k = [k_all[:, :, t:t + C].contiguous() for t in lens]
+    chunks_v = [v_all[:, :, t:t + C].contiguous() for t in lens]
 
     def run(dense):
+        ctx.zero_()
         for i in range(len(lens)):
-            chunk(i, dense)
+            api.quoka_append_kv(ps[i], chunks_k[i], chunks_v[i], k, v, None, ws)
+            if dense:
+                api.quoka_dense_chunk_attn(ps[i], q, k, v, out, None, ws)
+            else:
+                api.quoka_prefill_chunk(ps[i], q, k, v, out, None, None, ws)
+            ctx.add_(C)
 
     def timed(fn, reps):
         fn()
@@ -293,14 +476,13 @@ def sweep(args, w, q, k, v, out, ctx, dev, rank):
             ts.append(a.elapsed_time(b) * 1e3)
         return statistics.mean(ts)
 
+    k.zero_(); v.zero_()
     n0 = api.quoka_launch_count()
-    eager_us = timed(lambda: run(False), 5)
-    launches = (api.quoka_launch_count() - n0) // 6
-    per_chunk = []
-    for i in range(len(lens)):
-        per_chunk.append(round(timed(lambda: chunk(i, False), 3), 1))
+    eager_us = timed(lambda: run(False), 3)
+    launches = (api.quoka_launch_count() - n0) // 4
+    cache_ok = bool(torch.equal(k, k_all) and torch.equal(v, v_all))     # the loop rebuilt the whole cache
     dense_us = timed(lambda: run(True), 2)
-    graph_us = None
+    graph_us, graph_err = None, None
     try:
         g = torch.cuda.CUDAGraph()
         side = torch.cuda.Stream()
@@ -311,22 +493,67 @@ def sweep(args, w, q, k, v, out, ctx, dev, rank):
             with torch.cuda.graph(g, stream=side):
                 run(False)
         torch.cuda.synchronize()
-        graph_us = timed(g.replay, 5)
+        graph_us = timed(g.replay, 3)
     except Exception as e:                                      # capture not possible: report it, keep the eager number
-        graph_us = None
         graph_err = repr(e)[:200]
     status = api.quoka_last_device_status(ws)
     if rank == 0:
         line = {"metric": "us_per_prompt_prefill_attention", "value": round(eager_us, 1), "unit": "us",
                 "config": {"workload": args.workload, "chunks": len(lens), "chunk_len": C, "final_ctx_len": T,
-                           "budget_frac": frac, "n_retain": w["n_retain"]},
+                           "budget_frac": 0.12, "n_retain": w["n_retain"], "append": "quoka_append_kv per chunk"},
                 "sweep": {"quoka_eager_us": round(eager_us, 1), "quoka_graph_us": None if graph_us is None else round(graph_us, 1),
                           "dense_us": round(dense_us, 1), "speedup_vs_dense": round(dense_us / eager_us, 3),
-                          "per_chunk_us": per_chunk, "gpu_launches_per_sweep": launches},
+                          "us_per_chunk_eager": round(eager_us / len(lens), 2),
+                          "us_per_chunk_graph": None if graph_us is None else round(graph_us / len(lens), 2),
+                          "gpu_launches_per_sweep": launches, "cache_rebuilt_exactly": cache_ok},
                 "device_status": status, "note": "sweep mode (Algorithm 2 over the whole prompt); not the default bench line"}
-        if graph_us is None:
+        if graph_err:
             line["sweep"]["graph_error"] = graph_err
         print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------- timing grid at 32K context
+GRID = dict(budget_frac=(0.05, 0.12, 0.25, 0.5), C=(512, 2048, 8192), d=(64, 128), G=(1, 4, 8), n_retain=(32, 128, 512))
+
+
+def grid(args, dev, rank):
+    """The 4 x 3 x 2 x 3 x 3 = 216-point sweep at 32K cached context, 32 query heads: fused QuoKA chunk against the
+    dense chunk kernel, a few steps each, inputs drawn on the device (timing only; the parity of the sweep's
+    one-axis-at-a-time points and corners is a test)."""
+    from paper_2602_08722_b200 import api
+    T = 32768
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    rows = []
+    for C in GRID["C"]:
+        for d in GRID["d"]:
+            for G in GRID["G"]:
+                base = dict(batch=1, n_q=32, n_kv=32 // G, d=d, T=T, C=C, n_retain=128, kv_budget=0, budget_frac=0.12,
+                            dtype="bf16")
+                prob = Problem(base, args.seed, [T], dev, on_device=True)
+                ts = time_loop(prob.dense, 3, 1, lambda: flush_buf.fill_(1))
+                dense_us = statistics.mean(ts)
+                for frac in GRID["budget_frac"]:
+                    for N in GRID["n_retain"]:
+                        prob.p.budget_frac, prob.p.n_retain = frac, N
+                        prob.ws = api.alloc_workspace(prob.p)
+                        ts = time_loop(prob.step, 5, 2, lambda: flush_buf.fill_(1))
+                        us = statistics.mean(ts)
+                        rows.append({"budget_frac": frac, "chunk_len": C, "head_dim": d, "gqa": G, "n_retain": N,
+                                     "quoka_us": round(us, 1), "dense_us": round(dense_us, 1),
+                                     "speedup": round(dense_us / us, 2)})
+                st = api.quoka_last_device_status(prob.ws)
+                if st != 0:
+                    raise SystemExit(f"device status {st} at C={C} d={d} G={G}")
+                del prob
+                torch.cuda.empty_cache()
+    if rank == 0:
+        sp = [r["speedup"] for r in rows]
+        print(json.dumps({"metric": "grid_speedup_vs_dense_chunk_attn", "unit": "x", "points": len(rows),
+                          "value": round(statistics.median(sp), 2), "min": min(sp), "max": max(sp),
+                          "config": {"workload": "sweep_32k", "ctx_len": T, "n_q_heads": 32, "axes": {k: list(v) for k, v in GRID.items()},
+                                     "timing": "5 fused steps and 3 dense steps per point, CUDA events, L2 flushed between steps"},
+                          "rows": rows, "note": "grid mode; not the default bench line"}))
     return 0
 
 
@@ -340,14 +567,20 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the measurements of the other named workloads (the 'configs' object of the line)")
     ap.add_argument("--fused-only", action="store_true",
                     help="only the timed fused steps (for profiler captures): no per-kernel, e2e or CPU legs")
+    ap.add_argument("--stage", default=None, choices=["select_queries", "score_keys", "select_keys", "sparse_attn", "dense_attn"],
+                    help="with --fused-only: the timed steps call this one staged entry point instead of the fused call")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--cached-norms", action="store_true",
                     help="keep 1/|k| of every cache row beside the cache (quoka_update_key_norms) and let scoring read it")
     ap.add_argument("--sweep", action="store_true",
-                    help="chunked prefill of the whole prompt (Algorithm 2): chunks at cached lengths 0, C, 2C, .. T, "
-                         "eager launches and one CUDA graph, against the dense chunk kernel; prints its own JSON line")
+                    help="chunked prefill of the whole prompt (Algorithm 2 with a growing cache): chunks at cached lengths "
+                         "0, C, 2C, .. T, eager launches and one CUDA graph, against the dense chunk kernel; own JSON line")
+    ap.add_argument("--chunk", type=int, default=0, help="with --sweep: chunk length (default: the workload's)")
+    ap.add_argument("--grid", action="store_true", help="216-point timing sweep at 32K context; prints its own JSON line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -394,36 +627,18 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
 
-    inp = synth.make_chunk_inputs(rank_seed, w["batch"], w["n_q"], w["n_kv"], w["d"], ctx_lens, w["C"],
-                                  w["dtype"])
-    paged = bool(w.get("paged"))
-    if paged:
-        inp = synth.to_paged(inp, rank_seed)
-    q = inp.q.to(dev)
-    k = (inp.k_pages if paged else inp.k).to(dev)
-    v = (inp.v_pages if paged else inp.v).to(dev)
-    bt = inp.block_table.to(dev) if paged else None
-    ctx = inp.ctx_len.to(dev)
-    out = torch.zeros_like(q)
+    if args.grid:
+        return grid(args, dev, rank)
+    if args.sweep:
+        return sweep(args, w, dev, rank)
+
     impl = {"auto": api.IMPL_AUTO, "simt": api.IMPL_SIMT, "tensor": api.IMPL_TENSOR}[args.kernel_impl]
-    p = api.make_params(q, k, out, ctx, n_retain=w["n_retain"], kv_budget=w.get("kv_budget", 0),
-                        budget_frac=w.get("budget_frac", 0.0), max_ctx_len=max(ctx_lens), block_table=bt, impl=impl)
-    ws = api.alloc_workspace(p)
-    k_inv_norm = None
+    prob = Problem(w, rank_seed, ctx_lens, dev, impl=impl, cached_norms=args.cached_norms)
     if args.cached_norms:
-        k_inv_norm = torch.zeros(tuple(k.shape[:3]), dtype=torch.float32, device=dev)
-        api.quoka_update_key_norms(p, k, k_inv_norm, True, ws)
-        p.k_inv_norm = k_inv_norm.data_ptr()
         config["cached_key_norms"] = True
-    cap = api.quoka_kv_budget_cap(p)
+    p, q, k, v, out, ws, inp = prob.p, prob.q, prob.k, prob.v, prob.out, prob.ws, prob.inp
+    paged = prob.paged
     b, n_q, C, d = q.shape
-    n_kv = k.shape[1]
-    N = min(w["n_retain"], C)
-    q_idx = torch.zeros((b, n_q, N), dtype=torch.int32, device=dev)
-    qbar = torch.zeros((b, n_kv, N, d), dtype=q.dtype, device=dev)
-    scores = torch.zeros((b, n_kv, max(ctx_lens)), dtype=torch.float32, device=dev)
-    k_idx = torch.zeros((b, n_kv, cap), dtype=torch.int32, device=dev)
-    k_cnt = torch.zeros((b,), dtype=torch.int32, device=dev)
     flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
 
     def flush():
@@ -435,13 +650,14 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    if args.sweep:
-        return sweep(args, w, q, k, v, out, ctx, dev, rank)
+    step = prob.step
+    if args.fused_only and args.stage:
+        for fn in prob.stages().values():          # every stage once, so each has valid inputs
+            fn()
+        step = prob.dense if args.stage == "dense_attn" else prob.stages()[args.stage]
 
-    def step():
-        api.quoka_prefill_chunk(p, q, k, v, out, None, None, ws)
-
-    # ---- the timed region: exactly K fused steps
+    # ---- the timed region: exactly K fused steps.  The clock sampler keeps running through the per-kernel legs
+    # that feed the roofline figures.
     sampler = ClockSampler(local_rank)
     for _ in range(args.warmup):
         flush()
@@ -454,69 +670,25 @@ def main():
     barrier()
     t_wall = time.perf_counter() - t_wall
     launches = api.quoka_launch_count() - n0
-    clocks = sampler.stop()
     dev_status = api.quoka_last_device_status(ws)
     total_us = max_over_ranks(sum(per_step), world, dev)
     us_per_chunk = job_us_per_chunk(total_us, args.steps, world)
 
     if args.fused_only:
+        sampler.stop()
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": round(us_per_chunk, 2), "unit": UNIT, "n_gpus": world,
                               "steps": args.steps, "warmup": args.warmup, "config": config, "gpu_launches": launches,
+                              "stage": args.stage or "fused",
                               "note": "fused-only run (profiling aid); not a bench line"}))
         return 0
 
-    # ---- per-kernel timings: the staged entry points run back to back on the stream, exactly as the fused call
-    # issues them, with a CUDA event between stages (a kernel timed alone after an idle stream carries ~10 us of
-    # launch latency, which hides the small kernels); L2 is flushed before each sequence
-    ksteps = max(5, min(args.steps, 20))
-    stages = {
-        "select_queries": lambda: api.quoka_select_queries(p, q, q_idx, qbar, ws),
-        "score_keys": lambda: api.quoka_score_keys(p, qbar, k, scores, ws),
-        "select_keys": lambda: api.quoka_select_keys(p, scores, k_idx, k_cnt, ws),
-        "sparse_attn": lambda: api.quoka_sparse_attn(p, q, k, v, k_idx, k_cnt, out, None, ws),
-    }
-    work = sum_work(w, ctx_lens)
     pk = peaks()
-    samples = {name: [] for name in stages}
-    for it in range(ksteps + 3):
-        flush()
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)]
-        evs[0].record()
-        for i, fn in enumerate(stages.values()):
-            fn()
-            evs[i + 1].record()
-        torch.cuda.synchronize()
-        if it >= 3:
-            for i, name in enumerate(stages):
-                samples[name].append(evs[i].elapsed_time(evs[i + 1]) * 1e3)
-    kernels = {}
-    for name in stages:
-        ts = samples[name]
-        us = statistics.mean(ts)
-        kernels[name] = {"us": round(us, 2), "min_us": round(min(ts), 2),
-                         "gbs": round(work[name]["bytes"] / us / 1e3, 1),
-                         "tflops": round(work[name]["flops"] / us / 1e6, 2)}
-    dense_steps = 3 if work["dense_attn"]["flops"] > 2e12 else ksteps
-    ts = time_loop(lambda: api.quoka_dense_chunk_attn(p, q, k, v, out, None, ws), dense_steps, 1, flush)
-    us = statistics.mean(ts)
-    kernels["dense_attn"] = {"us": round(us, 2), "min_us": round(min(ts), 2),
-                             "gbs": round(work["dense_attn"]["bytes"] / us / 1e3, 1),
-                             "tflops": round(work["dense_attn"]["flops"] / us / 1e6, 2)}
-    for name, bound in (("select_queries", "hbm"), ("score_keys", "hbm"), ("select_keys", "hbm"),
-                        ("sparse_attn", "tensor"), ("dense_attn", "tensor")):
-        kk = kernels[name]
-        kk["bound"] = bound
-        kk["frac"] = round(kk["gbs"] / pk["hbm_gbs"], 4) if bound == "hbm" else round(kk["tflops"] / pk["bf16_tflops"], 4)
-    # scoring is tensor-bound once N exceeds the ridge point (flop per byte of K)
-    if work["score_keys"]["flops"] / (pk["bf16_tflops"] * 1e12) > work["score_keys"]["bytes"] / (pk["hbm_gbs"] * 1e9):
-        kernels["score_keys"]["bound"] = "tensor"
-        kernels["score_keys"]["frac"] = round(kernels["score_keys"]["tflops"] / pk["bf16_tflops"], 4)
-    staged_sum = sum(kernels[n]["us"] for n in stages)
+    kernels, staged_sum = per_kernel(prob, max(5, min(args.steps, 20)), flush, pk, args.workload)
+    clocks = sampler.stop()
     dom = "sparse_attn"
     roofline = {"kernel": dom, "bound": "tensor", "achieved": kernels[dom]["tflops"], "peak": pk["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": kernels[dom]["frac"],
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom)),
+                "unit": "TFLOP/s", "frac": kernels[dom]["frac"], "traffic": ncu_traffic(args.workload, dom),
                 "peak_source": f"{pk['source']} burst bf16 (kernel timed alone)"}
 
     # ---- end to end through the host-buffer entry point (contiguous caches only)
@@ -547,15 +719,24 @@ def main():
         cpu = {"value": round(us_cpu, 1), "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                "sample": sample, "cpu_seconds_spent": round(secs, 2)}
 
+    # ---- the other named workloads (one GPU only; after every timed region of the headline workload)
+    configs = None
+    if rank == 0 and world == 1 and not args.no_configs and args.workload == "llama8b_32k":
+        del prob, q, k, v, out, ws, p
+        torch.cuda.empty_cache()
+        configs = {}
+        for name, n_steps in (("long_128k", 10), ("serving_mix", 10), ("tiny_bf16", 20)):
+            configs[name] = side_config(name, args.seed, dev, flush, pk, n_steps, cpu_leg=not args.no_cpu_baseline)
+
     if rank == 0:
         line = {"metric": METRIC, "value": round(us_per_chunk, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": round(total_us / args.steps / 1e3, 4),
                 "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": w["dtype"],
                 "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
                 "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels,
-                "staged_sum_us": round(staged_sum, 2),
+                "staged_sum_us": staged_sum,
                 "speedup_vs_dense_chunk_attn": round(kernels["dense_attn"]["us"] / us_per_chunk / world, 3),
-                "device_status": dev_status, "wall_s_timed_region": round(t_wall, 3),
+                "device_status": dev_status, "wall_s_timed_region": round(t_wall, 3), "configs": configs,
                 "paper_context": "paper reports up to 5x attention speed-up at 30k tokens and 3x TTFT at 50k on A100 (ratios only)"}
         print(json.dumps(line))
     if world > 1:

@@ -110,9 +110,10 @@ __device__ __forceinline__ void resolve(AttnGeom& g, const int32_t* k_cnt, int s
 // rows first .. first + count - 1.  `diag` = chunk position of the tile's first row minus one tile-relative
 // offset, used by the causal limit: row r sees columns [0, r - col0 + 1).
 struct TileRows {
-  bool from_list;
+  bool from_list;       // addressing: rows list[first .. first + count), else the consecutive cache rows first ..
+  bool causal;          // masking: row r sees columns [0, r - col0 + 1), else columns [0, count)
   int first, count;     // consecutive rows (count may exceed the tile or be <= 0), or list base and remaining count
-  int col0;             // causal tiles: chunk position (dense: position in [0, T + C)) of column 0; list tiles: unused
+  int col0;             // causal tiles: chunk position (dense: position in [0, T + C)) of column 0
 };
 
 template <bool SPARSE>
@@ -122,12 +123,15 @@ __device__ __forceinline__ TileRows tile_rows(const AttnGeom& g, int t) {
     if (t < g.n_chunk) {
       const int ct = g.b_first ? (t == 0 ? g.c_a : t - 1) : t;
       r.from_list = false;
+      r.causal = true;
       r.first = g.T + ct * kKeyTile;
       r.count = g.C - ct * kKeyTile;
       r.col0 = ct * kKeyTile;
     } else {
+      // a list as long as the cache is the identity (the budget covers the cache): its tiles are plain row ranges
       const int st = t - g.n_chunk;
-      r.from_list = true;
+      r.from_list = g.cnt != g.T;
+      r.causal = false;
       r.first = st * kKeyTile;
       r.count = g.cnt - st * kKeyTile;
       r.col0 = 0;
@@ -135,6 +139,7 @@ __device__ __forceinline__ TileRows tile_rows(const AttnGeom& g, int t) {
   } else {
     const int j = g.n_dense - 1 - t;
     r.from_list = false;
+    r.causal = true;
     r.first = j * kKeyTile;
     r.count = g.T + g.C - j * kKeyTile;
     r.col0 = j * kKeyTile - g.T;            // chunk position of column 0 (negative inside the cache)
@@ -144,7 +149,7 @@ __device__ __forceinline__ TileRows tile_rows(const AttnGeom& g, int t) {
 
 // Number of visible columns of tile t for chunk row `row` (columns [0, lim) are visible).
 __device__ __forceinline__ int visible_cols(const TileRows& tr, int row) {
-  const int lim = tr.from_list ? tr.count : row - tr.col0 + 1;
+  const int lim = tr.causal ? row - tr.col0 + 1 : tr.count;
   return max(0, min(kKeyTile, lim));
 }
 
@@ -165,7 +170,8 @@ __device__ __forceinline__ float max32(uint32_t (&v)[32], bool masked, int col0,
 
 template <int HALVES, bool SPARSE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
-attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv_bfloat16* __restrict__ kc,
+attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const __nv_bfloat16* __restrict__ kc,
                const __nv_bfloat16* __restrict__ vc, const int32_t* __restrict__ k_idx,
                const int32_t* __restrict__ k_cnt, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
   constexpr int D = HALVES * 64;
@@ -203,6 +209,8 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
     mbar_init(q_full, 1);
     fence_mbar_init();
     tma_prefetch_desc(&tm_q);
+    tma_prefetch_desc(&tm_k);
+    tma_prefetch_desc(&tm_v);
   }
   if (warp == kMmaWarp) tmem_alloc(tmem_slot, 512);
   tc_fence_before();
@@ -402,6 +410,29 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __nv
 #pragma unroll 1
       for (int kvi = 0; kvi < 2; ++kvi) {                     // the tile's K rows, then its V rows
         if (!mbar_wait(&kv_empty[slot], phase ^ 1, wc)) { stop = true; break; }
+        // A whole tile of consecutive rows (page-aligned in a paged cache) is fetched by the copy engine as 64-row
+        // boxes: one thread issues them, the others only keep the barrier's arrival count.  Ragged tiles (rows past
+        // the end must read as zeros, not as whatever the cache holds there) and listed rows take the copies below.
+        if (!tr.from_list && tr.count >= kKeyTile && (P.page_size == 0 || (tr.first & (kPage - 1)) == 0)) {
+          if (lw == 0 && lane == 0) {
+            fence_proxy_async_smem();             // earlier contents of the slot were written through the generic proxy
+            mbar_arrive_expect_tx(&kv_full[slot], kTileBytes);
+            unsigned char* dst = kv_smem + (size_t)slot * kTileBytes;
+            const CUtensorMap* tm = kvi ? &tm_v : &tm_k;
+#pragma unroll
+            for (int sub = 0; sub < 2; ++sub) {
+              int c1 = tr.first + sub * 64, c3 = s;
+              if (P.page_size != 0) { c1 = 0; c3 = __ldg(table + (tr.first >> 6) + sub); }
+#pragma unroll
+              for (int hh = 0; hh < HALVES; ++hh)
+                tma_load_4d(dst + hh * kHalfBytes + sub * 64 * 128, tm, &kv_full[slot], hh * 64, c1, kv, c3);
+            }
+          } else {
+            mbar_arrive(&kv_full[slot]);
+          }
+          if (++slot == kSlots) { slot = 0; phase ^= 1; }
+          continue;
+        }
         if (kvi == 0 && tr.from_list && tile == g.n_chunk) list_rows(tr.first, tr.count);   // first list tile
         const uint4* src_base = reinterpret_cast<const uint4*>(kvi ? vc : kc);
         const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
@@ -566,6 +597,8 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
     const uint32_t box[4] = {64, 128, 1, 1};
     if (!encode_tensor_map_bf16(&tm_q, q, 4, dims, strides, box)) return QUOKA_ERR_CUDA;
   }
+  CUtensorMap tm_k, tm_v;
+  if (!encode_kv_tensor_map(&tm_k, p, k, 64) || !encode_kv_tensor_map(&tm_v, p, v, 64)) return QUOKA_ERR_CUDA;
   const int halves = P.d / 64;
   const size_t tile = (size_t)halves * 128 * 128;
   const size_t smem = 1024 + (2 + kSlots) * tile + 512;
@@ -592,7 +625,7 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
     attr[0].val.programmaticStreamSerializationAllowed = 1;                                                      \
     cfg.attrs = attr;                                                                                            \
     cfg.numAttrs = ((S) && after_selection) ? 1 : 0;                                                                                \
-    e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<H, S>, P, tm_q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, \
+    e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<H, S>, P, tm_q, tm_k, tm_v, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, \
                            k_idx, k_cnt, (__nv_bfloat16*)out, lse);                                              \
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                 \
   } while (0)

@@ -98,7 +98,7 @@ def attention_bound(out_oracle: np.ndarray, dtype: str) -> np.ndarray:
     bound = np.full(a.shape, mx)
     if dtype == "bf16":
         big = a >= 4.0
-        spacing = 2.0 ** (np.floor(np.log2(np.maximum(a, 4.0))) - 7)
+        spacing = np.ldexp(1.0, np.frexp(np.maximum(a, 4.0))[1] - 1 - 7)      # 2^(floor(log2 |o|) - 7), exactly
         bound = np.where(big, spacing / 2 + a * 2.0 ** -8, bound)
     return bound
 
