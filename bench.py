@@ -725,7 +725,8 @@ def main():
         del prob, q, k, v, out, ws, p
         torch.cuda.empty_cache()
         configs = {}
-        for name, n_steps in (("long_128k", 10), ("serving_mix", 10), ("tiny_bf16", 20)):
+        for name, n_steps in (("long_128k", 10), ("serving_mix", 10), ("tiny_bf16", 20), ("decode_32k", 20),
+                              ("decode_32k_b16", 20)):
             configs[name] = side_config(name, args.seed, dev, flush, pk, n_steps, cpu_leg=not args.no_cpu_baseline)
 
     if rank == 0:

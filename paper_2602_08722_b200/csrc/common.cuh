@@ -193,6 +193,14 @@ cudaError_t launch_select_keys(const DevParams& P, const float* scores, int32_t*
 cudaError_t launch_attn_simt(const DevParams& P, int dtype, const void* q, const void* k, const void* v,
                              const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st);
 
+// Generation phase (chunk of one query): matrix-vector scoring and a gather attention kernel.
+bool decode_path_applies(const DevParams& P);
+bool decode_attn_fits(const DevParams& P, bool with_list);
+cudaError_t launch_score_keys_gemv(const DevParams& P, int dtype, const void* qbar, const void* k, float* scores,
+                                   cudaStream_t st, bool chained);
+cudaError_t launch_decode_attn(const DevParams& P, int dtype, const void* q, const void* k, const void* v,
+                               const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
+                               bool chained);
 cudaError_t launch_append_kv(const DevParams& P, int dtype, const void* k_new, const void* v_new, void* k_cache,
                              void* v_cache, cudaStream_t st);
 

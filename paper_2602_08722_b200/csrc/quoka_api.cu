@@ -142,6 +142,10 @@ static quoka_status run_select_queries(const quoka_params* p, const DevParams& P
 static quoka_status run_score_keys(const quoka_params* p, const DevParams& P, const void* qbar, const void* k,
                                    float* scores, cudaStream_t st, bool chained = false) {
   if (p->max_ctx_len == 0) return QUOKA_OK;
+  if (p->impl == QUOKA_IMPL_AUTO && decode_path_applies(P)) {       // one query: a matrix-vector product
+    QUOKA_TRY_CUDA(launch_score_keys_gemv(P, p->dtype, qbar, k, scores, st, chained));
+    return QUOKA_OK;
+  }
   if (use_tensor(p) && score_keys_tc_supported(p)) return launch_score_keys_tc(p, P, qbar, k, scores, st, chained);
   if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;
   QUOKA_TRY_CUDA(launch_score_keys_simt(P, p->dtype, qbar, k, scores, st));
@@ -151,6 +155,10 @@ static quoka_status run_score_keys(const quoka_params* p, const DevParams& P, co
 static quoka_status run_attn(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                              const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                              bool after_selection = false) {
+  if (p->impl == QUOKA_IMPL_AUTO && P.chunk == 1 && decode_attn_fits(P, k_idx != nullptr)) {
+    QUOKA_TRY_CUDA(launch_decode_attn(P, p->dtype, q, k, v, k_idx, k_cnt, out, lse, st, after_selection));
+    return QUOKA_OK;
+  }
   if (use_tensor(p) && attn_tc_supported(p))
     return launch_attn_tc(p, P, q, k, v, k_idx, k_cnt, out, lse, st, after_selection);
   if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;

@@ -108,6 +108,33 @@ def test_decode_step_full_size_32k():
     check_chain(gp)
 
 
+@pytest.mark.parametrize("d,dtype", [(64, "bf16"), (128, "f32"), (64, "f32")])
+def test_decode_step_other_layouts_and_dense(d, dtype):
+    gp = problem(19, batch=2, n_q=8, n_kv=4, d=d, T=[1500, 77], C=1, dtype=dtype, n_retain=4, kv_budget=100)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(staged, gp.out)
+    # the same query over every cached row (Eq. 2)
+    api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+    torch.cuda.synchronize()
+    for s_ in range(gp.b):
+        q, k, v, T = gp.oracle_inputs(s_)
+        want, lse = O.dense_chunk_attention(q, k, v, T)
+        check_attention(f64(gp.out[s_]), want, dtype)
+        assert np.abs(f64(gp.lse[s_]) - lse).max() <= 2e-3
+
+
+def test_decode_step_with_more_listed_rows_than_the_gather_kernel_holds():
+    # 8500 listed rows + the query's own exceed the decode attention kernel's shared-memory logits: the general
+    # attention kernel takes over, the matrix-vector scoring stays
+    gp = problem(20, n_q=4, n_kv=2, T=9000, C=1, n_retain=4, kv_budget=8500)
+    gp.run_staged()
+    check_chain(gp)
+
+
 # ---------------------------------------------------------------- cached inverse key norms
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("paged", [False, True])
