@@ -392,8 +392,10 @@ def per_kernel(prob, ksteps, flush, pk, workload):
     kernels["dense_attn"] = {"us": round(us, 2), "min_us": round(min(ts), 2),
                              "gbs": round(work["dense_attn"]["bytes"] / us / 1e3, 1),
                              "tflops": round(work["dense_attn"]["flops"] / us / 1e6, 2)}
+    # one query per sequence: attention gathers B + 1 rows per head and is bound by memory latency / bandwidth
+    attn_bound = "hbm" if w["C"] == 1 else "tensor"
     for name, bound in (("select_queries", "hbm"), ("score_keys", "hbm"), ("select_keys", "hbm"),
-                        ("sparse_attn", "tensor"), ("dense_attn", "tensor")):
+                        ("sparse_attn", attn_bound), ("dense_attn", attn_bound)):
         kk = kernels[name]
         kk["bound"] = bound
         kk["frac"] = round(kk["gbs"] / pk["hbm_gbs"], 4) if bound == "hbm" else round(kk["tflops"] / pk["bf16_tflops"], 4)
