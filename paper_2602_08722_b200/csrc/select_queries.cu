@@ -1,15 +1,17 @@
 // Query sub-selection, normalisation and GQA pre-aggregation (Algorithm 1, first two blocks).
 //
-// rank_queries : a thread-block cluster of 8 CTAs per (sequence, query head); each CTA owns a
-//                contiguous slice of the head's C query rows.  Pass 1 reads the slice from HBM once
-//                (16-byte vector loads, D/8 lanes per row), keeps it in shared memory, and sums it
-//                into the CTA's share of the mean query; the shares are added across the cluster
-//                through distributed shared memory in a fixed order.  Pass 2 computes
-//                CosSim(q_r, M) for every row of the slice from shared memory, sorts the slice's
-//                (cosine, position) codes with a shared-memory bitonic sort, and places each of its
-//                N smallest by global rank: own rank + binary searches in the peers' sorted
-//                slices.  Codes are unique (the position is part of them), so the N lowest cosines
-//                come out in ascending order, equal cosines by position.
+// rank_queries : a thread-block cluster of 2 / 4 / 8 CTAs (by chunk length, about 256 rows per CTA) per
+//                (sequence, query head); each CTA owns a contiguous slice of the head's C query rows.
+//                Pass 1 brings the slice into shared memory with 16-byte cp.async in eight groups and sums
+//                the columns group by group as they land (a slice beyond the staging limit is re-read
+//                from L2 instead); the CTAs' shares of the mean query are added across the cluster
+//                through distributed shared memory in a fixed order.  Pass 2 computes CosSim(q_r, M) for
+//                every row of the slice (two lanes per row), packs (order code of the cosine, position)
+//                into one 64-bit key, sorts 32-key runs in registers (bitonic network over shuffles) and
+//                merges the runs by counting (branch-free binary searches, keys are unique).  Each CTA
+//                then copies the first codes of its peers' sorted slices into local shared memory and
+//                places each of its N smallest by global rank: own rank + number of smaller codes in
+//                every peer.  The N lowest cosines come out in ascending order, equal cosines by position.
 // aggregate    : one warp per (sequence, KV head, rank j): mean over the G heads of the group of
 //                their j-th retained query, each divided by its own norm; one rounding to dtype.
 #include <cooperative_groups.h>
