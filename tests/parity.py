@@ -5,7 +5,7 @@ oracle within that stage's tie rule, then the CUDA output itself (not the
 oracle's) is fed to the oracle's next stage.  Index work is bit-exact up to ties:
 a rank or a key may differ from the oracle's only where the oracle's own score
 gap is below 1e-4 relative.  Attention outputs on identical indices: bf16 within
-2e-2 max-abs (outputs below 4 in magnitude; see attention_bound for larger ones)
+2e-2 max-abs (outputs up to 3.1 in magnitude; see attention_bound for larger ones)
 and 2e-3 mean-abs; f32 within 2e-4 / 2e-5.
 """
 from __future__ import annotations
@@ -88,23 +88,22 @@ def check_key_selection(k_idx_gpu: np.ndarray, scores_oracle: np.ndarray, B: int
 def attention_bound(out_oracle: np.ndarray, dtype: str) -> np.ndarray:
     """Element-wise bound on |out_gpu - out_oracle|.
 
-    f32: 2e-4 everywhere.  bf16: the stated 2e-2 max-abs wherever |o| < 4.  An output of magnitude 4 or more is
-    STORED in bf16 with a spacing of 2^-5 or more, so rounding the exact result alone may cost half a spacing
-    (0.0156 for 4 <= |o| < 8) and leaves the arithmetic under 0.0044 of the 2e-2; there the bound is half a bf16
-    spacing of |o| plus 2^-8 |o| (bf16 softmax weights in the PV product: 2^-9 relative each, on a row dominated by
-    few keys they do not average out, and the row sum is taken before the rounding)."""
+    f32: 2e-4 everywhere.  bf16: the stated 2e-2 max-abs, or, where it is larger, what the arithmetic costs at
+    that magnitude: the output is STORED in bf16, so rounding the exact result alone may cost half a bf16 spacing
+    of |o| (0.0078 for 2 <= |o| < 4, 0.0156 for 4 <= |o| < 8), and the softmax weights enter the PV product as
+    bf16 (2^-9 relative each; on a row that few keys dominate they do not average out, and the row sum is taken
+    before the rounding), which adds up to 2^-8 |o|.  The sum exceeds 2e-2 from |o| = 3.12 on."""
     mx, _ = ATTN_TOL[dtype]
     a = np.abs(out_oracle)
     bound = np.full(a.shape, mx)
     if dtype == "bf16":
-        big = a >= 4.0
-        spacing = np.ldexp(1.0, np.frexp(np.maximum(a, 4.0))[1] - 1 - 7)      # 2^(floor(log2 |o|) - 7), exactly
-        bound = np.where(big, spacing / 2 + a * 2.0 ** -8, bound)
+        spacing = np.ldexp(1.0, np.frexp(np.maximum(a, 1.0))[1] - 1 - 7)      # 2^(floor(log2 |o|) - 7), exactly
+        bound = np.maximum(bound, spacing / 2 + a * 2.0 ** -8)
     return bound
 
 
 def check_attention(out_gpu: np.ndarray, out_oracle: np.ndarray, dtype: str):
-    """Returns the number of elements judged by the large-output bound (|o| >= 4, bf16 only)."""
+    """Returns the number of elements whose bound is above the stated 2e-2 (large outputs, bf16 only)."""
     diff = np.abs(out_gpu - out_oracle)
     _, mean = ATTN_TOL[dtype]
     assert np.isfinite(out_gpu).all()
@@ -113,7 +112,7 @@ def check_attention(out_gpu: np.ndarray, out_oracle: np.ndarray, dtype: str):
     assert (diff <= bound).all(), (f"attention abs diff {diff[worst]} > {bound[worst]} at {worst} "
                                    f"(oracle value {out_oracle[worst]})")
     assert diff.mean() <= mean, f"attention mean abs diff {diff.mean()} > {mean}"
-    return int((np.abs(out_oracle) >= 4.0).sum()) if dtype == "bf16" else 0
+    return int((bound > ATTN_TOL[dtype][0]).sum()) if dtype == "bf16" else 0
 
 
 class GpuProblem:
