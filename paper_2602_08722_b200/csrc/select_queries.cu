@@ -26,7 +26,9 @@ namespace quoka {
 
 constexpr int kRankThreads = 512;
 constexpr int kRankCluster = 8;
-constexpr size_t kRankStageLimit = 160 * 1024;   // a slice larger than this is re-read from L2 in pass 2
+// A slice larger than this is not kept in shared memory but re-read from L2 in pass 2: two CTAs must still fit an
+// SM (with 128 KB slices, chunk 4096, one CTA per SM meant two waves of the grid and a fifth more time).
+constexpr size_t kRankStageLimit = 84 * 1024;
 
 template <typename T> struct Raw8;                // 8 consecutive elements as 16-byte words
 template <> struct Raw8<__nv_bfloat16> { uint4 w[1]; };
