@@ -15,7 +15,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libquoka.so")
 LIB_DEBUG = os.path.join(PKG, "libquoka_debug.so")
 SOURCES = ["quoka_api.cu", "select_queries.cu", "score_keys_simt.cu", "score_keys_tc.cu", "select_keys.cu",
-           "attn_simt.cu", "attn_tc.cu", "no_alloc.cu", "cache_ops.cu", "diagnostics.cu", "decode.cu"]
+           "attn_simt.cu", "attn_tc.cu", "attn_tc_pair.cu", "no_alloc.cu", "cache_ops.cu", "diagnostics.cu", "decode.cu"]
 
 
 def _sources():

@@ -21,152 +21,9 @@
 // 384 threads and no register re-balancing between roles: every thread may use 168 registers
 // (with 512 threads and setmaxnreg the compiler still scheduled the softmax for 128 registers,
 // which halved its speed).
-#include "sm100_ptx.cuh"
-#include "tensor_kernels.cuh"
+#include "attn_tiles.cuh"
 
 namespace quoka {
-
-using namespace ptx;
-
-constexpr int kAttnThreads = 12 * 32;
-constexpr int kLoaderWarps = 3;
-constexpr int kMmaWarp = 11;
-constexpr int kQTile = 128;
-constexpr int kKeyTile = 128;
-constexpr int kSlots = 5;
-// The reference point m of the exponentials 2^(s - m) is raised, and O and l rescaled, only when a row's maximum
-// exceeds it by more than this many powers of two.  Until then P, l and O are simply larger by a common factor of at
-// most 2^32, which floating point carries without loss (bf16 and fp32 both reach 2^127; l <= 2^32 * keys and
-// |O| <= l * max|v| stay far below that); the quotient O / l does not change.  With 8 the rescale (a read-modify-
-// write of the whole accumulator row on the softmax -> PV chain) still ran often enough to cost 1-2 % of the kernel.
-constexpr float kRescaleThreshold = 32.0f;   // log2 units
-
-bool encode_kv_tensor_map(CUtensorMap* out, const quoka_params* p, const void* cache, uint32_t box_rows);
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// Every CTA walks ONE sequence of key tiles t = 0 .. n_total-1 for both of its Q tiles; Q tile x takes part in
-// the tiles t >= skip[x] (a suffix, so both finish on the same tile).
-//   dense : the tiles of rows [0, T + C) in DESCENDING order (the tiles only Q tile B sees come first).
-//   sparse: first the chunk's own tiles (the one only B sees, then tiles 0 .. c_a-1), THEN the tiles of the
-//           selected list.  The chunk's tiles do not depend on the key selection, so this kernel is launched
-//           with programmatic stream serialisation: it starts while the selection kernel still runs, works
-//           through the chunk tiles, and only then waits for the selection (`resolve`) to learn the list length.
-struct AttnGeom {
-  int T, C;
-  int n_chunk;        // sparse: tiles of the chunk's own rows in the sequence; dense: 0
-  int c_a;            // sparse: chunk tiles Q tile A sees
-  int b_first;        // sparse: 1 when the sequence starts with the tile only B sees
-  int skip_a;         // first tile Q tile A takes part in (B takes part in all); scalars, not arrays: the struct
-  bool active_b;      // must live in registers (an indexed member would put it in local memory)
-  int n_known;        // tiles known so far (sparse: n_chunk until resolved, then n_chunk + n_sel)
-  int cnt;            // sparse: selected rows (valid once resolved)
-  int n_dense;        // dense: number of tiles
-  bool resolved;
-};
-
-template <bool SPARSE>
-__device__ __forceinline__ AttnGeom make_geom(const DevParams& P, int s, int r0) {
-  AttnGeom g;
-  g.T = __ldg(P.ctx_len + s);
-  g.C = P.chunk;
-  const bool b_active = r0 + kQTile < g.C;
-  g.active_b = b_active;
-  g.cnt = 0;
-  if (SPARSE) {
-    g.c_a = r0 / kQTile + 1;
-    g.b_first = b_active ? 1 : 0;
-    g.n_chunk = g.c_a + g.b_first;
-    g.skip_a = g.b_first;
-    g.n_known = g.n_chunk;
-    g.n_dense = 0;
-    g.resolved = false;
-  } else {
-    const int last_a = min(r0 + kQTile - 1, g.C - 1), last_b = min(r0 + 2 * kQTile - 1, g.C - 1);
-    const int n_a = (g.T + last_a) / kKeyTile + 1;
-    const int n_b = b_active ? (g.T + last_b) / kKeyTile + 1 : 0;
-    g.n_dense = max(n_a, n_b);
-    g.skip_a = g.n_dense - n_a;
-    g.n_chunk = 0; g.c_a = 0; g.b_first = 0;
-    g.n_known = g.n_dense;
-    g.resolved = true;
-  }
-  return g;
-}
-
-// Sparse: wait for the selection kernel (a no-op when this kernel was not launched early) and read the list length.
-__device__ __forceinline__ void resolve(AttnGeom& g, const int32_t* k_cnt, int s) {
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  g.cnt = __ldcg(k_cnt + s);
-  g.n_known = g.n_chunk + (g.cnt + kKeyTile - 1) / kKeyTile;
-  g.resolved = true;
-}
-
-// Rows of tile t: from the selected list (`from_list`, rows list[base .. base + count)), or the consecutive cache
-// rows first .. first + count - 1.  `diag` = chunk position of the tile's first row minus one tile-relative
-// offset, used by the causal limit: row r sees columns [0, r - col0 + 1).
-struct TileRows {
-  bool from_list;       // addressing: rows list[first .. first + count), else the consecutive cache rows first ..
-  bool causal;          // masking: row r sees columns [0, r - col0 + 1), else columns [0, count)
-  int first, count;     // consecutive rows (count may exceed the tile or be <= 0), or list base and remaining count
-  int col0;             // causal tiles: chunk position (dense: position in [0, T + C)) of column 0
-};
-
-template <bool SPARSE>
-__device__ __forceinline__ TileRows tile_rows(const AttnGeom& g, int t) {
-  TileRows r;
-  if (SPARSE) {
-    if (t < g.n_chunk) {
-      const int ct = g.b_first ? (t == 0 ? g.c_a : t - 1) : t;
-      r.from_list = false;
-      r.causal = true;
-      r.first = g.T + ct * kKeyTile;
-      r.count = g.C - ct * kKeyTile;
-      r.col0 = ct * kKeyTile;
-    } else {
-      // a list as long as the cache is the identity (the budget covers the cache): its tiles are plain row ranges
-      const int st = t - g.n_chunk;
-      r.from_list = g.cnt != g.T;
-      r.causal = false;
-      r.first = st * kKeyTile;
-      r.count = g.cnt - st * kKeyTile;
-      r.col0 = 0;
-    }
-  } else {
-    const int j = g.n_dense - 1 - t;
-    r.from_list = false;
-    r.causal = true;
-    r.first = j * kKeyTile;
-    r.count = g.T + g.C - j * kKeyTile;
-    r.col0 = j * kKeyTile - g.T;            // chunk position of column 0 (negative inside the cache)
-  }
-  return r;
-}
-
-// Number of visible columns of tile t for chunk row `row` (columns [0, lim) are visible).
-__device__ __forceinline__ int visible_cols(const TileRows& tr, int row) {
-  const int lim = tr.causal ? row - tr.col0 + 1 : tr.count;
-  return max(0, min(kKeyTile, lim));
-}
-
-// Maximum of 32 score columns starting at col0; columns at and beyond `lim` are masked out.
-__device__ __forceinline__ float max32(uint32_t (&v)[32], bool masked, int col0, int lim) {
-  if (masked) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) if (col0 + i >= lim) v[i] = 0xFF800000u;    // -inf
-  }
-  float m0 = __uint_as_float(v[0]), m1 = __uint_as_float(v[1]);
-#pragma unroll
-  for (int i = 2; i < 30; i += 4) {
-    m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-    m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-  }
-  return max3(m0, m1, fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31])));
-}
 
 template <int HALVES, bool SPARSE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -590,6 +447,7 @@ bool attn_tc_supported(const quoka_params* p) {
 quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                             const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                             bool after_selection) {
+  if (attn_tc_pair_applies(P)) return launch_attn_tc_pair(p, P, q, k, v, k_idx, k_cnt, out, lse, st, after_selection);
   CUtensorMap tm_q;
   {
     const uint64_t dims[4] = {(uint64_t)P.d, (uint64_t)P.chunk, (uint64_t)P.n_q, (uint64_t)P.batch};

@@ -14,5 +14,10 @@ bool attn_tc_supported(const quoka_params* p);
 quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                             const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                             bool after_selection);
+// head_dim 128 with an even GQA ratio: the CTAs of two heads of a KV group work as a pair (cta_group::2)
+bool attn_tc_pair_applies(const DevParams& P);
+quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
+                                 const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
+                                 bool after_selection);
 
 }  // namespace quoka
