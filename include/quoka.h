@@ -118,7 +118,12 @@ quoka_status quoka_kv_budget_cap(const quoka_params* p, int32_t* cap);
 /* Bytes of workspace that every call below accepts (256-byte aligned pointer).
  * The first 256 bytes hold the device status word, which the caller sets to zero
  * once after allocating; the rest is scratch whose contents mean nothing between
- * calls.  Two calls that share a workspace must not overlap on the GPU. */
+ * calls.  Two calls that share a workspace must not overlap on the GPU.
+ * For problems whose attention grid is far smaller than the GPU (few heads, a short
+ * chunk) the size includes room for the partial results of the split attention
+ * kernel (each row block's keys are cut into up to 8 parts, one CTA each, and added
+ * up in part order: results are reproducible from run to run, and differ from the
+ * unsplit kernel's in the last bits only). */
 quoka_status quoka_workspace_size(const quoka_params* p, size_t* bytes);
 
 /* Alg. 1, "Query Sub-selection", then the normalisation and the mean over the G
@@ -210,9 +215,11 @@ quoka_status quoka_append_kv(const quoka_params* p, const void* k_new, const voi
  * array of QUOKA_STATIC_SCRATCH_BYTES that is part of the library image; every GPU that loads the
  * library holds that much memory until the process exits.  Inputs and outputs are still the
  * caller's.  The call allocates nothing and frees nothing.
- *   - Problems whose quoka_workspace_size exceeds QUOKA_STATIC_SCRATCH_BYTES are refused with
+ *   - Problems whose intermediates exceed QUOKA_STATIC_SCRATCH_BYTES are refused with
  *     QUOKA_ERR_STATIC_LIMIT before anything is launched (for scale: 32 q / 8 kv heads, d 128,
  *     131072 cached rows, N_Q 256 needs about 5.1 MiB; a batch of 8 at 65536 rows does not fit).
+ *     The array has no room for the split attention kernel's partial results: small grids run
+ *     unsplit here, so on those the output may differ from quoka_prefill_chunk's in the last bits.
  *   - The first call on each device looks up the array's device address (that device must be
  *     current); make that first call before any stream capture begins.
  *   - All calls in the process share the one array per device, and it keeps the previous call's

@@ -29,7 +29,7 @@ constexpr int kPairLoaderWarps = 3;
 constexpr uint32_t kPairSlotBytes = 16384;
 constexpr uint32_t kPairQTileBytes = 32768;
 
-template <bool SPARSE>
+template <bool SPARSE, bool SPLIT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kAttnThreads, 1)
 attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __nv_bfloat16* __restrict__ kc,
@@ -57,9 +57,22 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
   const WaitCtx wc{&abort_flag, P.status};
   const uint32_t rank = cluster_cta_rank();                   // 0: issues the MMAs; the pair is heads (2j, 2j + 1)
   const int s = blockIdx.z, h = blockIdx.x, kv = h / P.group;
-  const int rb = gridDim.y - 1 - blockIdx.y;                  // heaviest row blocks first
+  // grid.y = row blocks (heaviest first), times the parts a row block's key tiles are cut into (SPLIT)
+  const int n_parts = SPLIT ? P.attn_parts : 1;
+  const int n_rb = gridDim.y / n_parts;
+  const int rb = n_rb - 1 - blockIdx.y / n_parts;
   const int r0 = rb * 2 * kQTile;
   AttnGeom g = make_geom<SPARSE>(P, s, r0);
+  // SPLIT: this CTA walks the tiles [t_lo, t_hi) of the row block's sequence only and leaves, per row, a partial
+  // result (reference point, sum, un-normalised output); the part that finishes last adds the parts up.  The list
+  // length has to be known before the range is, so nothing of the walk starts before the selection has ended.
+  int t_lo = 0;
+  if (SPLIT) {
+    if (SPARSE) resolve(g, k_cnt, s);
+    const int part = blockIdx.y % n_parts;
+    t_lo = (int)(((long long)part * g.n_known) / n_parts);
+    g.n_known = (int)(((long long)(part + 1) * g.n_known) / n_parts);
+  }
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -97,8 +110,8 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
     float m_run = -INFINITY, l_run = 0.f;
     uint32_t phase = 0;
     bool ok = true;
-    const int skip_x = x ? 0 : g.skip_a;
-    const bool active_x = x ? g.active_b : true;
+    const int skip_x = max(x ? 0 : g.skip_a, t_lo);         // first tile this Q tile takes part in
+    const bool active_x = (x ? g.active_b : true) && (!SPLIT || skip_x < g.n_known);
     for (int t = skip_x; active_x; ++t) {
       if (t == g.n_known) {                                   // end of what is known: the list length, or the end
         if (g.resolved) break;
@@ -188,32 +201,112 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
       l_run += (ps0 + ps1) + (ps2 + ps3);
     }
     // ---- epilogue: O / l -> bf16 -> global
-    if (ok && active_x && mbar_wait(&o_full[x], 0, wc)) {
-      tc_fence_after();
-      const float inv = 1.f / l_run;
-      const bool store = row < P.chunk;
-      __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
+    if constexpr (!SPLIT) {
+      if (ok && active_x && mbar_wait(&o_full[x], 0, wc)) {
+        tc_fence_after();
+        const float inv = 1.f / l_run;
+        const bool store = row < P.chunk;
+        __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(o_addr + c * 32, r);
-        tmem_wait_ld();
-        if (store) {
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(o_addr + c * 32, r);
+          tmem_wait_ld();
+          if (store) {
 #pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint32_t w[4];
+            for (int v4 = 0; v4 < 4; ++v4) {
+              uint32_t w[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
-                                                               __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
-              w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+              for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
+                                                                 __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
+                w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+              }
+              *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
+        if (store && lse)
+          lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
       }
-      if (store && lse)
-        lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    } else {
+      // ---- this part's partial result (reference point m, sum l, un-normalised O; a part without tiles for this
+      // Q tile leaves m = -inf), then the merge by whichever part's warp arrives last.  One counter per (row block
+      // of a head, softmax warp); nobody waits for anybody.  The parts are added up in part order, so the result
+      // does not depend on which part came last.
+      constexpr int kTile = 130 * 128;                          // [128 columns of O | m | l][128 rows]
+      const int job = (s * P.n_q + h) * n_rb + rb;
+      const int part = blockIdx.y % n_parts;
+      float* tile0 = P.attn_partials + ((size_t)job * n_parts * 2 + x) * kTile;
+      float* mine = tile0 + (size_t)part * 2 * kTile;
+      const bool have = ok && active_x && mbar_wait(&o_full[x], 0, wc);
+      if (have) {
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(o_addr + c * 32, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mine[(c * 32 + i) * 128 + row_in_tile] = __uint_as_float(r[i]);
+        }
+      }
+      mine[128 * 128 + row_in_tile] = have ? m_run : -INFINITY;
+      mine[129 * 128 + row_in_tile] = have ? l_run : 0.f;
+      __threadfence();
+      __syncwarp();
+      int32_t* counter = P.attn_counters + (job * 2 + x) * 4 + quarter;
+      int arrived = 0;
+      if (lane == 0) arrived = atomicAdd(counter, 1);
+      arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
+      if (arrived == n_parts - 1) {
+        if (lane == 0) *counter = 0;                            // as the next launch expects it
+        __threadfence();
+        float wgt[8];
+        float M = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          wgt[q] = q < n_parts ? __ldcg(tile0 + (size_t)q * 2 * kTile + 128 * 128 + row_in_tile) : -INFINITY;
+          M = fmaxf(M, wgt[q]);
+        }
+        float l = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const float w = wgt[q] == -INFINITY ? 0.f : ex2(wgt[q] - M);
+          if (q < n_parts) l += w * __ldcg(tile0 + (size_t)q * 2 * kTile + 129 * 128 + row_in_tile);
+          wgt[q] = w;
+        }
+        const float inv = 1.f / l;
+        const bool store = row < P.chunk;
+        __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          float acc[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            if (q < n_parts && wgt[q] != 0.f) {
+              const float* src = tile0 + (size_t)q * 2 * kTile + (c * 32) * 128 + row_in_tile;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc[i] = fmaf(wgt[q], __ldcg(src + i * 128), acc[i]);
+            }
+          }
+          if (store) {
+#pragma unroll
+            for (int v4 = 0; v4 < 4; ++v4) {
+              uint32_t w[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] * inv, acc[v4 * 8 + 2 * i + 1] * inv);
+                w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+              }
+              *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        if (store && lse) lse[((long long)s * P.n_q + h) * P.chunk + row] = (M + log2f(l)) * 0.6931471805599453f;
+      }
     }
   } else if (warp < 8 + kPairLoaderWarps) {
     // ================================================================== K / V loaders: this CTA's half of every tile
@@ -339,14 +432,14 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
       if (++slot == kPairSlots) { slot = 0; phase ^= 1; }
       return true;
     };
-    for (int tile = 0;; ++tile) {
+    for (int tile = t_lo;; ++tile) {
       if (tile == g.n_known) {                                // end of what is known: the list length, or the end
         if (g.resolved) break;
         resolve(g, k_cnt, s);
         if (tile == g.n_known) break;
       }
       const TileRows tr = tile_rows<SPARSE>(g, tile);
-      const bool first_list_tile = tr.from_list && tile == g.n_chunk;
+      const bool first_list_tile = tr.from_list && tile == max(g.n_chunk, t_lo);
       if (!item(std::false_type{}, tr, first_list_tile)) break;
       if (!item(std::true_type{}, tr, first_list_tile)) break;
     }
@@ -364,7 +457,7 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
       const uint32_t peer_full0 = map_to_cta(smem_u32(peer_full), 0);
       int slot = 0;
       uint32_t phase = 0;
-      for (int tile = 0; ok; ++tile) {
+      for (int tile = t_lo; ok; ++tile) {
         if (tile == g.n_known) {
           if (g.resolved) break;
           resolve(g, k_cnt, s);
@@ -432,27 +525,27 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
       // Tile t: O += P_t V_t for each Q tile taking part (as the two halves of P arrive), then S = Q K_{t+1}^T.
       // K_{t+1} and V_t are both acquired before the P waits, so those never sit on the P -> PV -> QK chain.
       const auto part = [&](int x, int t) { return x ? g.active_b : t >= g.skip_a; };
-      if (ok) {
+      if (ok && t_lo < g.n_known) {
         k_slot = acquire();
         if (ok) {
-          if (part(0, 0)) issue_qk(0, k_slot);
-          if (part(1, 0)) issue_qk(1, k_slot);
+          if (part(0, t_lo)) issue_qk(0, k_slot);
+          if (part(1, t_lo)) issue_qk(1, k_slot);
           mma_pair_commit(&kv_empty[k_slot]);
         }
-        for (int t = 0; ok; ++t) {
+        for (int t = t_lo; ok; ++t) {
           if (t + 1 == g.n_known && !g.resolved) resolve(g, k_cnt, s);
           const bool more = t + 1 < g.n_known;
           v_slot = acquire();
           if (ok && more) k_slot = acquire();
           if (!ok) break;
           if (part(0, t)) {
-            issue_pv(0, v_slot, t == g.skip_a);
+            issue_pv(0, v_slot, t == max(g.skip_a, t_lo));
             if (!ok) break;
             if (!more) mma_pair_commit(&o_full[0]);
           }
           if (more && part(0, t + 1)) issue_qk(0, k_slot);
           if (part(1, t)) {
-            issue_pv(1, v_slot, t == 0);
+            issue_pv(1, v_slot, t == t_lo);
             if (!ok) break;
             if (!more) mma_pair_commit(&o_full[1]);
           }
@@ -472,6 +565,34 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
 // ---------------------------------------------------------------------------------------------- host
 bool attn_tc_pair_applies(const DevParams& P) { return P.d == 128 && P.group % 2 == 0; }
 
+// Split attention.  A grid of fewer CTAs than half the SMs (short chunks, few heads) leaves most of the GPU idle
+// while every CTA walks its whole key sequence; cutting each row block's tiles into parts fills it.  A part costs a
+// start-up and a pass over the partial results, so parts keep at least six tiles.
+static int pair_sm_count() {
+  static int n = []() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return v;
+  }();
+  return n;
+}
+static long long pair_jobs(const quoka_params* p) {
+  return (long long)p->n_q_heads * ((p->chunk_len + 2 * kQTile - 1) / (2 * kQTile)) * p->batch;
+}
+int attn_split_parts(const quoka_params* p, int tiles) {
+  if (p->dtype != QUOKA_BF16 || p->head_dim != 128 || (p->n_q_heads / p->n_kv_heads) % 2 != 0) return 1;
+  const long long jobs = pair_jobs(p);
+  long long parts = pair_sm_count() / jobs;
+  if (parts > tiles / 6) parts = tiles / 6;
+  if (parts > 8) parts = 8;
+  return parts < 1 ? 1 : (int)parts;
+}
+size_t attn_split_partial_bytes(const quoka_params* p, int parts) {
+  return parts <= 1 ? 0 : (size_t)pair_jobs(p) * parts * 2 * 130 * 128 * sizeof(float);
+}
+size_t attn_split_counter_bytes(const quoka_params* p) { return (size_t)pair_jobs(p) * 8 * sizeof(int32_t); }
+
 quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                                  const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                                  bool after_selection) {
@@ -485,15 +606,23 @@ quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, cons
   CUtensorMap tm_k, tm_v;
   if (!encode_kv_tensor_map(&tm_k, p, k, 64) || !encode_kv_tensor_map(&tm_v, p, v, 64)) return QUOKA_ERR_CUDA;
   const size_t smem = 1024 + 2 * kPairQTileBytes + (size_t)kPairSlots * kPairSlotBytes + 512;
-  dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.batch);   // n_q is even: clusters of (2, 1, 1)
   const bool sparse = k_idx != nullptr;
+  // key tiles of the longest row block this call can meet (the list or the cache, plus the chunk's own)
+  const int tiles = ((sparse ? P.budget_cap : P.max_ctx) + kKeyTile - 1) / kKeyTile + 1;
+  const int parts = P.attn_partials ? attn_split_parts(p, tiles) : 1;
+  DevParams PP = P;
+  PP.attn_parts = parts;
+  dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile) * parts, P.batch);   // n_q is even: clusters of (2, 1, 1)
+  if (parts > 1 && !after_selection &&          // (the fused call clears the counters before its first kernel)
+      cudaMemsetAsync(P.attn_counters, 0, attn_split_counter_bytes(p), st) != cudaSuccess)
+    return QUOKA_ERR_CUDA;
   log_launch(sparse ? "attn_tc_pair<sparse>" : "attn_tc_pair<dense>", grid, dim3(kAttnThreads), smem, 2,
              sparse && after_selection);
   cudaError_t e = cudaSuccess;
   // Programmatic stream serialisation inside the fused call only, as for the one-CTA kernel.
-#define QUOKA_ATTN_PAIR(S)                                                                                        \
+#define QUOKA_ATTN_PAIR(S, X)                                                                                      \
   do {                                                                                                            \
-    e = cudaFuncSetAttribute(attn_tc_pair_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
+    e = cudaFuncSetAttribute(attn_tc_pair_kernel<S, X>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                  \
     cudaLaunchConfig_t cfg = {};                                                                                  \
     cfg.gridDim = grid;                                                                                           \
@@ -505,11 +634,12 @@ quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;                                                       \
     cfg.attrs = attr;                                                                                             \
     cfg.numAttrs = ((S) && after_selection) ? 1 : 0;                                                              \
-    e = cudaLaunchKernelEx(&cfg, attn_tc_pair_kernel<S>, P, tm_q, tm_k, tm_v, (const __nv_bfloat16*)k,            \
+    e = cudaLaunchKernelEx(&cfg, attn_tc_pair_kernel<S, X>, PP, tm_q, tm_k, tm_v, (const __nv_bfloat16*)k,        \
                            (const __nv_bfloat16*)v, k_idx, k_cnt, (__nv_bfloat16*)out, lse);                      \
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                  \
   } while (0)
-  if (sparse) QUOKA_ATTN_PAIR(true); else QUOKA_ATTN_PAIR(false);
+  if (parts > 1) { if (sparse) QUOKA_ATTN_PAIR(true, true); else QUOKA_ATTN_PAIR(false, true); }
+  else { if (sparse) QUOKA_ATTN_PAIR(true, false); else QUOKA_ATTN_PAIR(false, false); }
 #undef QUOKA_ATTN_PAIR
   count_launch();
   return cudaGetLastError() == cudaSuccess ? QUOKA_OK : QUOKA_ERR_CUDA;

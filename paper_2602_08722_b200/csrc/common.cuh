@@ -34,6 +34,10 @@ struct DevParams {
   int agg_mean;     // 1: mean over the retained queries instead of the maximum
   const float* k_inv_norm;  // cached 1/|k| per cache row, or null
   int64_t kv_rows;  // rows per (sequence, head) when contiguous
+  // split attention (small grids): room for the parts' partial results and their arrival counters, or null
+  float* attn_partials;
+  int32_t* attn_counters;
+  int attn_parts;   // parts per row block of the launch at hand (set by the launcher), 1 = no split
 };
 
 // B_s of one sequence: min(B_SA, T) or floor(frac*T + 0.5) in double.
@@ -207,6 +211,11 @@ cudaError_t launch_append_kv(const DevParams& P, int dtype, const void* k_new, c
 // Host checks shared by the fused entry points (everything but the workspace); nothing is enqueued before they pass.
 quoka_status check_prefill_args(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
                                 const void* out);
+// the fused call behind quoka_prefill_chunk, and its workspace need, with or without the split-attention scratch
+quoka_status prefill_chunk_impl(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache, void* out,
+                                int32_t* k_idx_out, int32_t* k_cnt_out, void* ws, size_t ws_bytes, void* stream,
+                                bool with_split);
+size_t workspace_bytes(const quoka_params* p, bool with_split);
 // Device address of the built-in scratch array on the current device (looked up once per device).
 quoka_status static_scratch_for_current_device(void** out);
 

@@ -44,14 +44,13 @@ extern "C" quoka_status quoka_prefill_chunk_static(const quoka_params* p, const 
   // every host-side refusal comes before the first thing put on the stream (the memset below)
   quoka_status st = quoka::check_prefill_args(p, q, k_cache, v_cache, out);
   if (st != QUOKA_OK) return st;
-  size_t need = 0;
-  if ((st = quoka_workspace_size(p, &need)) != QUOKA_OK) return st;
-  if (need > (size_t)QUOKA_STATIC_SCRATCH_BYTES) return QUOKA_ERR_STATIC_LIMIT;
+  // the array has no room for the scratch of the split attention kernel: small grids run unsplit here
+  if (quoka::workspace_bytes(p, /*with_split=*/false) > (size_t)QUOKA_STATIC_SCRATCH_BYTES) return QUOKA_ERR_STATIC_LIMIT;
   void* scratch = nullptr;
   if ((st = quoka::static_scratch_for_current_device(&scratch)) != QUOKA_OK) return st;
   // The array keeps whatever the previous call left.  Only the status word has to start at zero;
   // everything else is written before it is read.
   if (cudaMemsetAsync(scratch, 0, 256, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QUOKA_ERR_CUDA;
-  return quoka_prefill_chunk(p, q, k_cache, v_cache, out, k_idx_out, k_cnt_out, scratch,
-                             (size_t)QUOKA_STATIC_SCRATCH_BYTES, stream);
+  return quoka::prefill_chunk_impl(p, q, k_cache, v_cache, out, k_idx_out, k_cnt_out, scratch,
+                                   (size_t)QUOKA_STATIC_SCRATCH_BYTES, stream, /*with_split=*/false);
 }

@@ -22,6 +22,8 @@ struct Workspace {
   float* scores;
   int32_t* k_idx;
   int32_t* k_cnt;
+  float* attn_partials;      // split attention of small grids: partial results and arrival counters, or null
+  int32_t* attn_counters;
   size_t total;
 };
 
@@ -30,7 +32,16 @@ static int budget_cap_of(const quoka_params* p) {
   return cap < 1 ? 1 : cap;
 }
 
-static Workspace carve(const quoka_params* p, void* ws) {
+// Parts the attention kernels may cut a row block into for this problem (the larger of the sparse and the dense call's).
+static int attn_parts_bound(const quoka_params* p) {
+  if (p->impl == QUOKA_IMPL_SIMT || p->chunk_len <= 1) return 1;
+  const int cap = budget_cap_of(p);
+  const int sparse = attn_split_parts(p, (cap + 127) / 128 + 1), dense = attn_split_parts(p, (p->max_ctx_len + 127) / 128 + 1);
+  return sparse > dense ? sparse : dense;
+}
+
+// with_split = false: the layout without the split-attention scratch (every call still works, small grids unsplit)
+static Workspace carve(const quoka_params* p, void* ws, bool with_split = true) {
   Workspace w{};
   const size_t es = p->dtype == QUOKA_BF16 ? 2 : 4;
   const int N = p->n_retain < p->chunk_len ? p->n_retain : p->chunk_len;
@@ -48,6 +59,11 @@ static Workspace carve(const quoka_params* p, void* ws) {
   w.scores = reinterpret_cast<float*>(take((size_t)p->batch * p->n_kv_heads * (size_t)(p->max_ctx_len > 0 ? p->max_ctx_len : 1) * 4));
   w.k_idx = reinterpret_cast<int32_t*>(take((size_t)p->batch * p->n_kv_heads * cap * 4));
   w.k_cnt = reinterpret_cast<int32_t*>(take((size_t)p->batch * 4));
+  const int parts = with_split ? attn_parts_bound(p) : 1;
+  if (parts > 1) {
+    w.attn_counters = reinterpret_cast<int32_t*>(take(attn_split_counter_bytes(p)));
+    w.attn_partials = reinterpret_cast<float*>(take(attn_split_partial_bytes(p, parts)));
+  }
   w.total = off;
   return w;
 }
@@ -92,13 +108,15 @@ quoka_status check_prefill_args(const quoka_params* p, const void* q, const void
   return QUOKA_OK;
 }
 
-static quoka_status check_ws(const quoka_params* p, void* ws, size_t ws_bytes) {
+static quoka_status check_ws(const quoka_params* p, void* ws, size_t ws_bytes, bool with_split = true) {
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0) return QUOKA_ERR_WORKSPACE;
-  if (ws_bytes < carve(p, nullptr).total) return QUOKA_ERR_WORKSPACE;
+  if (ws_bytes < carve(p, nullptr, with_split).total) return QUOKA_ERR_WORKSPACE;
   return QUOKA_OK;
 }
 
-static DevParams make_dev(const quoka_params* p, void* ws) {
+size_t workspace_bytes(const quoka_params* p, bool with_split) { return carve(p, nullptr, with_split).total; }
+
+static DevParams make_dev(const quoka_params* p, void* ws, bool with_split = true) {
   DevParams P{};
   P.batch = p->batch; P.n_q = p->n_q_heads; P.n_kv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
   P.d = p->head_dim; P.chunk = p->chunk_len; P.n_retain = p->n_retain;
@@ -116,6 +134,8 @@ static DevParams make_dev(const quoka_params* p, void* ws) {
   P.agg_mean = p->query_agg == QUOKA_AGG_MEAN ? 1 : 0;
   P.k_inv_norm = p->k_inv_norm;
   P.kv_rows = p->kv_rows;
+  const Workspace w = carve(p, ws, with_split);
+  P.attn_partials = w.attn_partials; P.attn_counters = w.attn_counters; P.attn_parts = 1;
   return P;
 }
 
@@ -164,6 +184,31 @@ static quoka_status run_attn(const quoka_params* p, const DevParams& P, const vo
   if (p->impl == QUOKA_IMPL_TENSOR) return QUOKA_ERR_UNSUPPORTED;
   QUOKA_TRY_CUDA(launch_attn_simt(P, p->dtype, q, k, v, k_idx, k_cnt, out, lse, st));
   return QUOKA_OK;
+}
+
+// The fused loop body.  with_split = false keeps to the workspace layout without the split-attention scratch (the
+// built-in array of the no-allocation entry point has no room for it).
+quoka_status prefill_chunk_impl(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache, void* out,
+                                int32_t* k_idx_out, int32_t* k_cnt_out, void* ws, size_t ws_bytes, void* stream,
+                                bool with_split) {
+  quoka_status st = check_prefill_args(p, q, k_cache, v_cache, out);
+  if (st != QUOKA_OK) return st;
+  if ((st = check_ws(p, ws, ws_bytes, with_split)) != QUOKA_OK) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  DevParams P = make_dev(p, ws, with_split);
+  Workspace w = carve(p, ws, with_split);
+  int32_t* k_idx = k_idx_out ? k_idx_out : w.k_idx;
+  int32_t* k_cnt = k_cnt_out ? k_cnt_out : w.k_cnt;
+  // the split attention's arrival counters start at zero; cleared here so that nothing sits between the selection
+  // kernel and the attention kernel on the stream
+  if (w.attn_counters) QUOKA_TRY_CUDA(cudaMemsetAsync(w.attn_counters, 0, attn_split_counter_bytes(p), cs));
+  if (p->max_ctx_len > 0) {
+    if ((st = run_select_queries(p, P, q, w.q_idx, w.qbar, cs)) != QUOKA_OK) return st;
+    if ((st = run_score_keys(p, P, w.qbar, k_cache, w.scores, cs, /*chained=*/true)) != QUOKA_OK) return st;
+  }
+  // with an empty cache the selection kernel only writes k_cnt = 0 and the -1 padding
+  QUOKA_TRY_CUDA(launch_select_keys(P, w.scores, k_idx, k_cnt, cs, /*chained=*/p->max_ctx_len > 0));
+  return run_attn(p, P, q, k_cache, v_cache, k_idx, k_cnt, out, nullptr, cs, /*after_selection=*/true);
 }
 
 }  // namespace quoka
@@ -252,21 +297,7 @@ quoka_status quoka_dense_chunk_attn(const quoka_params* p, const void* q, const 
 quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache,
                                  void* out, int32_t* k_idx_out, int32_t* k_cnt_out, void* ws, size_t ws_bytes,
                                  void* stream) {
-  quoka_status st = check_prefill_args(p, q, k_cache, v_cache, out);
-  if (st != QUOKA_OK) return st;
-  if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
-  cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  DevParams P = make_dev(p, ws);
-  Workspace w = carve(p, ws);
-  int32_t* k_idx = k_idx_out ? k_idx_out : w.k_idx;
-  int32_t* k_cnt = k_cnt_out ? k_cnt_out : w.k_cnt;
-  if (p->max_ctx_len > 0) {
-    if ((st = run_select_queries(p, P, q, w.q_idx, w.qbar, cs)) != QUOKA_OK) return st;
-    if ((st = run_score_keys(p, P, w.qbar, k_cache, w.scores, cs, /*chained=*/true)) != QUOKA_OK) return st;
-  }
-  // with an empty cache the selection kernel only writes k_cnt = 0 and the -1 padding
-  QUOKA_TRY_CUDA(launch_select_keys(P, w.scores, k_idx, k_cnt, cs, /*chained=*/p->max_ctx_len > 0));
-  return run_attn(p, P, q, k_cache, v_cache, k_idx, k_cnt, out, nullptr, cs, /*after_selection=*/true);
+  return prefill_chunk_impl(p, q, k_cache, v_cache, out, k_idx_out, k_cnt_out, ws, ws_bytes, stream, /*with_split=*/true);
 }
 
 quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_len_host, const void* q_host,

@@ -16,6 +16,11 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
                             bool after_selection);
 // head_dim 128 with an even GQA ratio: the CTAs of two heads of a KV group work as a pair (cta_group::2)
 bool attn_tc_pair_applies(const DevParams& P);
+// Small grids: the key tiles of every row block are cut into this many parts, one CTA each (1 = no split).
+// `tiles` = key tiles of the longest row block the call can meet.  Scratch for the partial results:
+int attn_split_parts(const quoka_params* p, int tiles);
+size_t attn_split_partial_bytes(const quoka_params* p, int parts);
+size_t attn_split_counter_bytes(const quoka_params* p);
 quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                                  const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                                  bool after_selection);

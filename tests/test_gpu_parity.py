@@ -497,3 +497,41 @@ def test_back_to_back_fused_calls_when_the_budget_covers_every_cache(C, T):
     for o, i, c in zip(outs, idxs, cnts):
         assert torch.equal(o, want) and torch.equal(i, want_idx) and torch.equal(c, gp.k_cnt)
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+# ------------------------------------------------------------------ split attention (grids far smaller than the GPU)
+# With few heads and a short chunk the tensor-core attention kernel cuts every row block's key tiles into parts, one
+# CTA each; the parts leave partial results (reference point, sum, un-normalised output) and whichever finishes last
+# adds them up in part order.  Shapes below: 8 query heads x 1 row block x batch = 8..16 CTAs before the split, 29-33
+# key tiles, so four parts; a short sequence next to a long one gives parts with no tile at all.
+@pytest.mark.gpu
+@pytest.mark.parametrize("paged", [False, True])
+@pytest.mark.parametrize("T,C", [(4100, 200), ([4100, 300], 129), ([3000, 0, 4000], 256)])
+def test_split_attention_sparse_against_the_oracle(T, C, paged):
+    batch = len(T) if isinstance(T, list) else 1
+    gp = problem(31, batch=batch, n_q=8, n_kv=2, T=T, C=C, n_retain=16, kv_budget=0, budget_frac=0.9, paged=paged)
+    gp.run_staged()
+    check_chain(gp)          # every row of every head, lse included
+    staged = gp.out.clone()
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged)          # same parts, added in the same order
+    assert api.quoka_last_device_status(gp.ws) == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("T,C", [(4100, 200), ([4100, 300], 129)])
+def test_split_attention_dense_against_the_oracle(T, C):
+    batch = len(T) if isinstance(T, list) else 1
+    gp = problem(32, batch=batch, n_q=8, n_kv=2, T=T, C=C)
+    for rep in range(2):     # twice: the arrival counters must be back at zero after a launch
+        gp.out.zero_()
+        api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+        torch.cuda.synchronize()
+        for s in range(batch):
+            q, k, v, Ts = gp.oracle_inputs(s)
+            want, lse = O.dense_chunk_attention(q, k, v, Ts)
+            check_attention(f64(gp.out[s]), want, "bf16")
+            assert np.abs(f64(gp.lse[s]) - lse).max() <= 2e-3
+    assert api.quoka_last_device_status(gp.ws) == 0
