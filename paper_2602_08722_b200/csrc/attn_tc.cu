@@ -25,7 +25,7 @@
 
 namespace quoka {
 
-template <int HALVES, bool SPARSE>
+template <int HALVES, bool SPARSE, bool SPLIT>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __nv_bfloat16* __restrict__ kc,
@@ -54,9 +54,22 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
   // grid = (heads, row blocks, batch): heads vary fastest so the CTAs resident together share a KV head's
   // rows in L2, and the row blocks run heaviest (most causal tiles) first, lightest last
   const int s = blockIdx.z, h = blockIdx.x, kv = h / P.group;
-  const int rb = gridDim.y - 1 - blockIdx.y;
+  // (SPLIT: grid.y = row blocks times the parts a row block's key tiles are cut into)
+  const int n_parts = SPLIT ? P.attn_parts : 1;
+  const int n_rb = gridDim.y / n_parts;
+  const int rb = n_rb - 1 - blockIdx.y / n_parts;
   const int r0 = rb * 2 * kQTile;
   AttnGeom g = make_geom<SPARSE>(P, s, r0);
+  // SPLIT: this CTA walks the tiles [t_lo, t_hi) of the row block's sequence only and leaves, per row, a partial
+  // result; the part that finishes last adds the parts up.  The list length has to be known before the range is, so
+  // nothing of the walk starts before the selection has ended.
+  int t_lo = 0;
+  if (SPLIT) {
+    if (SPARSE) resolve(g, k_cnt, s);
+    const int part = blockIdx.y % n_parts;
+    t_lo = (int)(((long long)part * g.n_known) / n_parts);
+    g.n_known = (int)(((long long)(part + 1) * g.n_known) / n_parts);
+  }
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -87,8 +100,8 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
     float m_run = -INFINITY, l_run = 0.f;
     uint32_t phase = 0;
     bool ok = true;
-    const int skip_x = x ? 0 : g.skip_a;
-    const bool active_x = x ? g.active_b : true;
+    const int skip_x = max(x ? 0 : g.skip_a, t_lo);         // first tile this Q tile takes part in
+    const bool active_x = (x ? g.active_b : true) && (!SPLIT || skip_x < g.n_known);
     for (int t = skip_x; active_x; ++t) {
       if (t == g.n_known) {                                   // end of what is known: the list length, or the end
         if (g.resolved) break;
@@ -183,32 +196,39 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
       l_run += (ps0 + ps1) + (ps2 + ps3);
     }
     // ---- epilogue: O / l -> bf16 -> global
-    if (ok && active_x && mbar_wait(&o_full[x], 0, wc)) {
-      tc_fence_after();
-      const float inv = 1.f / l_run;
-      const bool store = row < P.chunk;
-      __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
+    if constexpr (!SPLIT) {
+      if (ok && active_x && mbar_wait(&o_full[x], 0, wc)) {
+        tc_fence_after();
+        const float inv = 1.f / l_run;
+        const bool store = row < P.chunk;
+        __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(o_addr + c * 32, r);
-        tmem_wait_ld();
-        if (store) {
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(o_addr + c * 32, r);
+          tmem_wait_ld();
+          if (store) {
 #pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint32_t w[4];
+            for (int v4 = 0; v4 < 4; ++v4) {
+              uint32_t w[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
-                                                               __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
-              w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+              for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
+                                                                 __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
+                w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+              }
+              *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
+        if (store && lse)
+          lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
       }
-      if (store && lse)
-        lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    } else {
+      const bool have = ok && active_x && mbar_wait(&o_full[x], 0, wc);
+      if (have) tc_fence_after();
+      attn_split_epilogue<D>(P, (s * P.n_q + h) * n_rb + rb, blockIdx.y % n_parts, n_parts, x, quarter, lane, row_in_tile, row, have,
+                             o_addr, m_run, l_run, s, h, out, lse);
     }
   } else if (warp < 8 + kLoaderWarps) {
     // ================================================================== K / V row loaders (gather)
@@ -256,7 +276,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
     };
 #pragma unroll
     for (int k = 0; k < LIST_REGS; ++k) t_list[k] = -1;
-    for (int tile = 0;; ++tile) {
+    for (int tile = t_lo;; ++tile) {
       if (tile == g.n_known) {                                // end of what is known: the list length, or the end
         if (g.resolved) break;
         resolve(g, k_cnt, s);
@@ -290,7 +310,7 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
           if (++slot == kSlots) { slot = 0; phase ^= 1; }
           continue;
         }
-        if (kvi == 0 && tr.from_list && tile == g.n_chunk) list_rows(tr.first, tr.count);   // first list tile
+        if (kvi == 0 && tr.from_list && tile == max(g.n_chunk, t_lo)) list_rows(tr.first, tr.count);   // first list tile
         const uint4* src_base = reinterpret_cast<const uint4*>(kvi ? vc : kc);
         const uint32_t dst_tile = kv_base + slot * kTileBytes + (c16 >> 3) * kHalfBytes;
         int t[RPT];                                               // row number, or -1
@@ -399,27 +419,27 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
     // K_{t+1} and V_t are both acquired before the P waits, so those never sit on the P -> PV -> QK chain.
     // The sparse sequence's length is learnt (resolve) just before the look-ahead past the chunk's own tiles.
     const auto part = [&](int x, int t) { return x ? g.active_b : t >= g.skip_a; };
-    if (ok) {
+    if (ok && t_lo < g.n_known) {
       k_slot = acquire();
       if (ok) {
-        if (part(0, 0)) issue_qk(0, k_slot);
-        if (part(1, 0)) issue_qk(1, k_slot);
+        if (part(0, t_lo)) issue_qk(0, k_slot);
+        if (part(1, t_lo)) issue_qk(1, k_slot);
         mma_commit(&kv_empty[k_slot]);
       }
-      for (int t = 0; ok; ++t) {
+      for (int t = t_lo; ok; ++t) {
         if (t + 1 == g.n_known && !g.resolved) resolve(g, k_cnt, s);
         const bool more = t + 1 < g.n_known;
         v_slot = acquire();
         if (ok && more) k_slot = acquire();
         if (!ok) break;
         if (part(0, t)) {
-          issue_pv(0, v_slot, t == g.skip_a);
+          issue_pv(0, v_slot, t == max(g.skip_a, t_lo));
           if (!ok) break;
           if (!more) mma_commit(&o_full[0]);
         }
         if (more && part(0, t + 1)) issue_qk(0, k_slot);
         if (part(1, t)) {
-          issue_pv(1, v_slot, t == 0);
+          issue_pv(1, v_slot, t == t_lo);
           if (!ok) break;
           if (!more) mma_commit(&o_full[1]);
         }
@@ -436,6 +456,40 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
 }
 
 // ---------------------------------------------------------------------------------------------- host
+// Split attention.  A grid of fewer CTAs than half the SMs (short chunks, few heads) leaves most of the GPU idle
+// while every CTA walks its whole key sequence; cutting each row block's tiles into parts fills it.  A part costs a
+// start-up and a pass over the partial results, so parts keep at least six tiles.
+static int attn_sm_count() {
+  static int n = []() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return v;
+  }();
+  return n;
+}
+static long long attn_jobs(const quoka_params* p) {
+  return (long long)p->n_q_heads * ((p->chunk_len + 2 * kQTile - 1) / (2 * kQTile)) * p->batch;
+}
+int attn_split_parts(const quoka_params* p, int tiles) {
+  if (p->dtype != QUOKA_BF16) return 1;
+  const long long jobs = attn_jobs(p);
+  long long parts = attn_sm_count() / jobs;
+  if (parts > tiles / 6) parts = tiles / 6;
+  if (parts > 8) parts = 8;
+  return parts < 1 ? 1 : (int)parts;
+}
+size_t attn_split_partial_bytes(const quoka_params* p, int parts) {
+  return parts <= 1 ? 0 : (size_t)attn_jobs(p) * parts * 2 * kSplitTileFloats * sizeof(float);
+}
+size_t attn_split_counter_bytes(const quoka_params* p) { return (size_t)attn_jobs(p) * 8 * sizeof(int32_t); }
+// Parts of the launch at hand: `tiles` = key tiles of the longest row block the call can meet (the list or the
+// cache, plus the chunk's own).  Without room for the partial results (the no-allocation entry point) nothing splits.
+int attn_split_parts_for_launch(const quoka_params* p, const DevParams& P, bool sparse) {
+  if (!P.attn_partials) return 1;
+  return attn_split_parts(p, ((sparse ? P.budget_cap : P.max_ctx) + kKeyTile - 1) / kKeyTile + 1);
+}
+
 bool attn_tc_supported(const quoka_params* p) {
   if (p->dtype != QUOKA_BF16) return false;
   // the loaders address cache rows in 32-bit units of 16 bytes
@@ -460,8 +514,14 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
   const int halves = P.d / 64;
   const size_t tile = (size_t)halves * 128 * 128;
   const size_t smem = 1024 + (2 + kSlots) * tile + 512;
-  dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile), P.batch);
   const bool sparse = k_idx != nullptr;
+  const int parts = attn_split_parts_for_launch(p, P, sparse);
+  DevParams PP = P;
+  PP.attn_parts = parts;
+  dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile) * parts, P.batch);
+  if (parts > 1 && !after_selection &&          // (the fused call clears the counters before its first kernel)
+      cudaMemsetAsync(P.attn_counters, 0, attn_split_counter_bytes(p), st) != cudaSuccess)
+    return QUOKA_ERR_CUDA;
   log_launch(sparse ? "attn_tc<sparse>" : "attn_tc<dense>", grid, dim3(kAttnThreads), smem, 1, sparse && after_selection);
   cudaError_t e = cudaSuccess;
   // Inside the fused call the sparse kernel is launched with programmatic stream serialisation: it may start
@@ -469,9 +529,9 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
   // kernel's other inputs) still runs; it touches the selection's outputs only after its own
   // griddepcontrol.wait.  A stand-alone call keeps the ordinary stream order: whatever ran before it may have
   // written q, k or v.
-#define QUOKA_ATTN_TC(H, S)                                                                                      \
+#define QUOKA_ATTN_TC(H, S, X)                                                                                   \
   do {                                                                                                           \
-    e = cudaFuncSetAttribute(attn_tc_kernel<H, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
+    e = cudaFuncSetAttribute(attn_tc_kernel<H, S, X>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                 \
     cudaLaunchConfig_t cfg = {};                                                                                 \
     cfg.gridDim = grid;                                                                                          \
@@ -483,12 +543,17 @@ quoka_status launch_attn_tc(const quoka_params* p, const DevParams& P, const voi
     attr[0].val.programmaticStreamSerializationAllowed = 1;                                                      \
     cfg.attrs = attr;                                                                                            \
     cfg.numAttrs = ((S) && after_selection) ? 1 : 0;                                                                                \
-    e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<H, S>, P, tm_q, tm_k, tm_v, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, \
+    e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<H, S, X>, PP, tm_q, tm_k, tm_v, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, \
                            k_idx, k_cnt, (__nv_bfloat16*)out, lse);                                              \
     if (e != cudaSuccess) return QUOKA_ERR_CUDA;                                                                 \
   } while (0)
-  if (halves == 2) { if (sparse) QUOKA_ATTN_TC(2, true); else QUOKA_ATTN_TC(2, false); }
-  else { if (sparse) QUOKA_ATTN_TC(1, true); else QUOKA_ATTN_TC(1, false); }
+  if (parts > 1) {
+    if (halves == 2) { if (sparse) QUOKA_ATTN_TC(2, true, true); else QUOKA_ATTN_TC(2, false, true); }
+    else { if (sparse) QUOKA_ATTN_TC(1, true, true); else QUOKA_ATTN_TC(1, false, true); }
+  } else {
+    if (halves == 2) { if (sparse) QUOKA_ATTN_TC(2, true, false); else QUOKA_ATTN_TC(2, false, false); }
+    else { if (sparse) QUOKA_ATTN_TC(1, true, false); else QUOKA_ATTN_TC(1, false, false); }
+  }
 #undef QUOKA_ATTN_TC
   count_launch();
   return cudaGetLastError() == cudaSuccess ? QUOKA_OK : QUOKA_ERR_CUDA;

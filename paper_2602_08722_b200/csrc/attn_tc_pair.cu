@@ -230,83 +230,10 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
           lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
       }
     } else {
-      // ---- this part's partial result (reference point m, sum l, un-normalised O; a part without tiles for this
-      // Q tile leaves m = -inf), then the merge by whichever part's warp arrives last.  One counter per (row block
-      // of a head, softmax warp); nobody waits for anybody.  The parts are added up in part order, so the result
-      // does not depend on which part came last.
-      constexpr int kTile = 130 * 128;                          // [128 columns of O | m | l][128 rows]
-      const int job = (s * P.n_q + h) * n_rb + rb;
-      const int part = blockIdx.y % n_parts;
-      float* tile0 = P.attn_partials + ((size_t)job * n_parts * 2 + x) * kTile;
-      float* mine = tile0 + (size_t)part * 2 * kTile;
       const bool have = ok && active_x && mbar_wait(&o_full[x], 0, wc);
-      if (have) {
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(o_addr + c * 32, r);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mine[(c * 32 + i) * 128 + row_in_tile] = __uint_as_float(r[i]);
-        }
-      }
-      mine[128 * 128 + row_in_tile] = have ? m_run : -INFINITY;
-      mine[129 * 128 + row_in_tile] = have ? l_run : 0.f;
-      __threadfence();
-      __syncwarp();
-      int32_t* counter = P.attn_counters + (job * 2 + x) * 4 + quarter;
-      int arrived = 0;
-      if (lane == 0) arrived = atomicAdd(counter, 1);
-      arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
-      if (arrived == n_parts - 1) {
-        if (lane == 0) *counter = 0;                            // as the next launch expects it
-        __threadfence();
-        float wgt[8];
-        float M = -INFINITY;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          wgt[q] = q < n_parts ? __ldcg(tile0 + (size_t)q * 2 * kTile + 128 * 128 + row_in_tile) : -INFINITY;
-          M = fmaxf(M, wgt[q]);
-        }
-        float l = 0.f;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const float w = wgt[q] == -INFINITY ? 0.f : ex2(wgt[q] - M);
-          if (q < n_parts) l += w * __ldcg(tile0 + (size_t)q * 2 * kTile + 129 * 128 + row_in_tile);
-          wgt[q] = w;
-        }
-        const float inv = 1.f / l;
-        const bool store = row < P.chunk;
-        __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          float acc[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            if (q < n_parts && wgt[q] != 0.f) {
-              const float* src = tile0 + (size_t)q * 2 * kTile + (c * 32) * 128 + row_in_tile;
-#pragma unroll
-              for (int i = 0; i < 32; ++i) acc[i] = fmaf(wgt[q], __ldcg(src + i * 128), acc[i]);
-            }
-          }
-          if (store) {
-#pragma unroll
-            for (int v4 = 0; v4 < 4; ++v4) {
-              uint32_t w[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] * inv, acc[v4 * 8 + 2 * i + 1] * inv);
-                w[i] = *reinterpret_cast<const uint32_t*>(&b2);
-              }
-              *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          }
-        }
-        if (store && lse) lse[((long long)s * P.n_q + h) * P.chunk + row] = (M + log2f(l)) * 0.6931471805599453f;
-      }
+      if (have) tc_fence_after();
+      attn_split_epilogue<D>(P, (s * P.n_q + h) * n_rb + rb, blockIdx.y % n_parts, n_parts, x, quarter, lane, row_in_tile, row, have,
+                             o_addr, m_run, l_run, s, h, out, lse);
     }
   } else if (warp < 8 + kPairLoaderWarps) {
     // ================================================================== K / V loaders: this CTA's half of every tile
@@ -565,34 +492,6 @@ attn_tc_pair_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const
 // ---------------------------------------------------------------------------------------------- host
 bool attn_tc_pair_applies(const DevParams& P) { return P.d == 128 && P.group % 2 == 0; }
 
-// Split attention.  A grid of fewer CTAs than half the SMs (short chunks, few heads) leaves most of the GPU idle
-// while every CTA walks its whole key sequence; cutting each row block's tiles into parts fills it.  A part costs a
-// start-up and a pass over the partial results, so parts keep at least six tiles.
-static int pair_sm_count() {
-  static int n = []() {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return v;
-  }();
-  return n;
-}
-static long long pair_jobs(const quoka_params* p) {
-  return (long long)p->n_q_heads * ((p->chunk_len + 2 * kQTile - 1) / (2 * kQTile)) * p->batch;
-}
-int attn_split_parts(const quoka_params* p, int tiles) {
-  if (p->dtype != QUOKA_BF16 || p->head_dim != 128 || (p->n_q_heads / p->n_kv_heads) % 2 != 0) return 1;
-  const long long jobs = pair_jobs(p);
-  long long parts = pair_sm_count() / jobs;
-  if (parts > tiles / 6) parts = tiles / 6;
-  if (parts > 8) parts = 8;
-  return parts < 1 ? 1 : (int)parts;
-}
-size_t attn_split_partial_bytes(const quoka_params* p, int parts) {
-  return parts <= 1 ? 0 : (size_t)pair_jobs(p) * parts * 2 * 130 * 128 * sizeof(float);
-}
-size_t attn_split_counter_bytes(const quoka_params* p) { return (size_t)pair_jobs(p) * 8 * sizeof(int32_t); }
-
 quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                                  const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                                  bool after_selection) {
@@ -607,9 +506,7 @@ quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, cons
   if (!encode_kv_tensor_map(&tm_k, p, k, 64) || !encode_kv_tensor_map(&tm_v, p, v, 64)) return QUOKA_ERR_CUDA;
   const size_t smem = 1024 + 2 * kPairQTileBytes + (size_t)kPairSlots * kPairSlotBytes + 512;
   const bool sparse = k_idx != nullptr;
-  // key tiles of the longest row block this call can meet (the list or the cache, plus the chunk's own)
-  const int tiles = ((sparse ? P.budget_cap : P.max_ctx) + kKeyTile - 1) / kKeyTile + 1;
-  const int parts = P.attn_partials ? attn_split_parts(p, tiles) : 1;
+  const int parts = attn_split_parts_for_launch(p, P, sparse);
   DevParams PP = P;
   PP.attn_parts = parts;
   dim3 grid(P.n_q, (P.chunk + 2 * kQTile - 1) / (2 * kQTile) * parts, P.batch);   // n_q is even: clusters of (2, 1, 1)

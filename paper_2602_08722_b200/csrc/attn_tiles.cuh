@@ -149,4 +149,89 @@ __device__ __forceinline__ float max32(uint32_t (&v)[32], bool masked, int col0,
   return max3(m0, m1, fmaxf(__uint_as_float(v[30]), __uint_as_float(v[31])));
 }
 
+// ---------------------------------------------------------------------------------------------- split attention
+// A launch whose grid is far smaller than the GPU cuts every row block's key tiles into parts, one CTA (pair) each.
+constexpr int kSplitTileFloats = 130 * 128;     // one part's partial result of a 128-row Q tile
+
+// Epilogue of a softmax warp of a split launch.
+template <int D>
+__device__ __forceinline__ void attn_split_epilogue(const DevParams& P, int job, int part, int n_parts, int x, int quarter,
+                                                    int lane, int row_in_tile, int row, bool have, uint32_t o_addr,
+                                                    float m_run, float l_run, int s, int h, __nv_bfloat16* out,
+                                                    float* lse) {
+  // ---- this part's partial result (reference point m, sum l, un-normalised O; a part without tiles for this
+  // Q tile leaves m = -inf), then the merge by whichever part's warp arrives last.  One counter per (row block
+  // of a head, softmax warp); nobody waits for anybody.  The parts are added up in part order, so the result
+  // does not depend on which part came last.
+  constexpr int kTile = kSplitTileFloats;                   // [D columns of O | m | l][128 rows], D <= 128
+  float* tile0 = P.attn_partials + ((size_t)job * n_parts * 2 + x) * kTile;
+  float* mine = tile0 + (size_t)part * 2 * kTile;
+  if (have) {
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t r[32];
+      tmem_ld32(o_addr + c * 32, r);
+      tmem_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) mine[(c * 32 + i) * 128 + row_in_tile] = __uint_as_float(r[i]);
+    }
+  }
+  mine[D * 128 + row_in_tile] = have ? m_run : -INFINITY;
+  mine[(D + 1) * 128 + row_in_tile] = have ? l_run : 0.f;
+  __threadfence();
+  __syncwarp();
+  int32_t* counter = P.attn_counters + (job * 2 + x) * 4 + quarter;
+  int arrived = 0;
+  if (lane == 0) arrived = atomicAdd(counter, 1);
+  arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
+  if (arrived == n_parts - 1) {
+    if (lane == 0) *counter = 0;                            // as the next launch expects it
+    __threadfence();
+    float wgt[8];
+    float M = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      wgt[q] = q < n_parts ? __ldcg(tile0 + (size_t)q * 2 * kTile + D * 128 + row_in_tile) : -INFINITY;
+      M = fmaxf(M, wgt[q]);
+    }
+    float l = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float w = wgt[q] == -INFINITY ? 0.f : ex2(wgt[q] - M);
+      if (q < n_parts) l += w * __ldcg(tile0 + (size_t)q * 2 * kTile + (D + 1) * 128 + row_in_tile);
+      wgt[q] = w;
+    }
+    const float inv = 1.f / l;
+    const bool store = row < P.chunk;
+    __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+      float acc[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (q < n_parts && wgt[q] != 0.f) {
+          const float* src = tile0 + (size_t)q * 2 * kTile + (c * 32) * 128 + row_in_tile;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = fmaf(wgt[q], __ldcg(src + i * 128), acc[i]);
+        }
+      }
+      if (store) {
+#pragma unroll
+        for (int v4 = 0; v4 < 4; ++v4) {
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[v4 * 8 + 2 * i] * inv, acc[v4 * 8 + 2 * i + 1] * inv);
+            w[i] = *reinterpret_cast<const uint32_t*>(&b2);
+          }
+          *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+    if (store && lse) lse[((long long)s * P.n_q + h) * P.chunk + row] = (M + log2f(l)) * 0.6931471805599453f;
+  }
+}
+
 }  // namespace quoka

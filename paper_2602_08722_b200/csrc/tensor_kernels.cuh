@@ -21,6 +21,7 @@ bool attn_tc_pair_applies(const DevParams& P);
 int attn_split_parts(const quoka_params* p, int tiles);
 size_t attn_split_partial_bytes(const quoka_params* p, int parts);
 size_t attn_split_counter_bytes(const quoka_params* p);
+int attn_split_parts_for_launch(const quoka_params* p, const DevParams& P, bool sparse);
 quoka_status launch_attn_tc_pair(const quoka_params* p, const DevParams& P, const void* q, const void* k, const void* v,
                                  const int32_t* k_idx, const int32_t* k_cnt, void* out, float* lse, cudaStream_t st,
                                  bool after_selection);

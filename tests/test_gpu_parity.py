@@ -535,3 +535,26 @@ def test_split_attention_dense_against_the_oracle(T, C):
             check_attention(f64(gp.out[s]), want, "bf16")
             assert np.abs(f64(gp.lse[s]) - lse).max() <= 2e-3
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,n_q,n_kv", [(64, 8, 2), (128, 4, 4), (128, 6, 2)])
+def test_split_attention_in_the_one_cta_kernel(d, n_q, n_kv):
+    # head_dim 64, one query head per KV head, an odd GQA ratio: the shapes the CTA-pair kernel does not take
+    gp = problem(33, batch=2, n_q=n_q, n_kv=n_kv, d=d, T=[4100, 300], C=200, n_retain=16, kv_budget=0, budget_frac=0.9)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged)
+    for s in range(2):
+        gp.out.zero_()
+        api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+        torch.cuda.synchronize()
+        q, k, v, Ts = gp.oracle_inputs(s)
+        want, lse = O.dense_chunk_attention(q, k, v, Ts)
+        check_attention(f64(gp.out[s]), want, "bf16")
+        assert np.abs(f64(gp.lse[s]) - lse).max() <= 2e-3
+    assert api.quoka_last_device_status(gp.ws) == 0
