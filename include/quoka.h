@@ -194,7 +194,15 @@ quoka_status quoka_prefill_chunk(const quoka_params* p, const void* q, const voi
  * cache, runs quoka_prefill_chunk, and copies out_dev -> out_host
  * ([b][n_Q][C][d] dense), all on `stream`.  ctx_len_host is a HOST copy of T_s.
  * Paged caches are not supported here (QUOKA_ERR_UNSUPPORTED).  q_dev / out_dev
- * must be dense [b][n_Q][C][d] and p's q/o strides must describe them. */
+ * must be dense [b][n_Q][C][d] and p's q/o strides must describe them.
+ * A chunk of 8 MiB of queries or more is cut into 2 or 4 slices of whole KV
+ * groups, and slice i+1 is copied in and slice i-1 copied out on two streams of
+ * the library's own (made on first use, one set per device) while slice i is
+ * computed on `stream`; the result is the same bits as the unsliced call's.
+ * Towards `stream` the call is still ordered like one operation (it forks from
+ * `stream` at its start and joins it at its end, also under stream capture).
+ * Two such calls must not overlap on one device (they share the side streams
+ * and their events), whatever streams they are given. */
 quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_len_host,
                                       const void* q_host, const void* k_new_host, const void* v_new_host,
                                       void* out_host, void* q_dev, void* k_cache, void* v_cache, void* out_dev,

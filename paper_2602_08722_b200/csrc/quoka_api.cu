@@ -5,6 +5,8 @@
 #include <cstdio>
 #include <cstdlib>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "tensor_kernels.cuh"
 
@@ -186,6 +188,35 @@ static quoka_status run_attn(const quoka_params* p, const DevParams& P, const vo
   return QUOKA_OK;
 }
 
+// Two side streams and the events that tie them to the caller's stream, made once per device: the host-buffer entry
+// point brings the next slice of a chunk in and takes the previous one out while the current one is computed.
+struct HostPipe {
+  cudaStream_t h2d = nullptr, d2h = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, in[4] = {}, done[4] = {};
+  bool ok = false, tried = false;
+};
+static HostPipe* host_pipe_for_current_device() {
+  constexpr int kMaxDev = 64;
+  static HostPipe pipes[kMaxDev];
+  static std::mutex mu;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  HostPipe& hp = pipes[dev];
+  if (!hp.tried) {
+    hp.tried = true;
+    bool good = cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaEventCreateWithFlags(&hp.fork, cudaEventDisableTiming) == cudaSuccess &&
+                cudaEventCreateWithFlags(&hp.join, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 4 && good; ++i)
+      good = cudaEventCreateWithFlags(&hp.in[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming) == cudaSuccess;
+    hp.ok = good;
+  }
+  return hp.ok ? &hp : nullptr;
+}
+
 // The fused loop body.  with_split = false keeps to the workspace layout without the split-attention scratch (the
 // built-in array of the no-allocation entry point has no room for it).
 quoka_status prefill_chunk_impl(const quoka_params* p, const void* q, const void* k_cache, const void* v_cache, void* out,
@@ -320,21 +351,74 @@ quoka_status quoka_prefill_chunk_host(const quoka_params* p, const int32_t* ctx_
     if (ctx_len_host[s] < 0 || ctx_len_host[s] > p->max_ctx_len) return QUOKA_ERR_INVALID_ARG;
   if ((st = check_ws(p, ws, ws_bytes)) != QUOKA_OK) return st;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  const size_t q_bytes = (size_t)p->batch * p->n_q_heads * C * d * es;
-  QUOKA_TRY_CUDA(cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, cs));
-  for (int s = 0; s < p->batch; ++s) {
-    const size_t dst_off = ((size_t)s * p->kv_stride_b + (size_t)ctx_len_host[s] * p->kv_stride_t) * es;
-    const size_t src_off = (size_t)s * p->n_kv_heads * C * d * es;
-    QUOKA_TRY_CUDA(cudaMemcpy2DAsync(static_cast<char*>(k_cache) + dst_off, (size_t)p->kv_stride_h * es,
-                                     static_cast<const char*>(k_new_host) + src_off, (size_t)C * d * es,
-                                     (size_t)C * d * es, p->n_kv_heads, cudaMemcpyHostToDevice, cs));
-    QUOKA_TRY_CUDA(cudaMemcpy2DAsync(static_cast<char*>(v_cache) + dst_off, (size_t)p->kv_stride_h * es,
-                                     static_cast<const char*>(v_new_host) + src_off, (size_t)C * d * es,
-                                     (size_t)C * d * es, p->n_kv_heads, cudaMemcpyHostToDevice, cs));
+  // Copies of the KV heads [kv0, kv0 + n_kv) and their query heads; every (sequence, head) block is contiguous on
+  // both sides, the sequences are `pitch` apart.
+  const int G = p->n_q_heads / p->n_kv_heads;
+  const size_t head_bytes = (size_t)C * d * es;
+  auto copy_in = [&](int kv0, int n_kv, cudaStream_t on) -> cudaError_t {
+    cudaError_t e = cudaMemcpy2DAsync(static_cast<char*>(q_dev) + (size_t)kv0 * G * head_bytes, (size_t)p->q_stride_b * es,
+                                      static_cast<const char*>(q_host) + (size_t)kv0 * G * head_bytes,
+                                      (size_t)p->n_q_heads * head_bytes, (size_t)n_kv * G * head_bytes, p->batch,
+                                      cudaMemcpyHostToDevice, on);
+    for (int s = 0; s < p->batch && e == cudaSuccess; ++s) {
+      const size_t dst_off = ((size_t)s * p->kv_stride_b + (size_t)kv0 * p->kv_stride_h + (size_t)ctx_len_host[s] * p->kv_stride_t) * es;
+      const size_t src_off = ((size_t)s * p->n_kv_heads + kv0) * head_bytes;
+      e = cudaMemcpy2DAsync(static_cast<char*>(k_cache) + dst_off, (size_t)p->kv_stride_h * es,
+                            static_cast<const char*>(k_new_host) + src_off, head_bytes, head_bytes, n_kv,
+                            cudaMemcpyHostToDevice, on);
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(static_cast<char*>(v_cache) + dst_off, (size_t)p->kv_stride_h * es,
+                              static_cast<const char*>(v_new_host) + src_off, head_bytes, head_bytes, n_kv,
+                              cudaMemcpyHostToDevice, on);
+    }
+    return e;
+  };
+  auto copy_out = [&](int kv0, int n_kv, cudaStream_t on) -> cudaError_t {
+    return cudaMemcpy2DAsync(static_cast<char*>(out_host) + (size_t)kv0 * G * head_bytes, (size_t)p->n_q_heads * head_bytes,
+                             static_cast<const char*>(out_dev) + (size_t)kv0 * G * head_bytes, (size_t)p->o_stride_b * es,
+                             (size_t)n_kv * G * head_bytes, p->batch, cudaMemcpyDeviceToHost, on);
+  };
+  // A large chunk is cut into slices of whole KV groups (the selection and the attention of a KV group need nothing
+  // of another group): slice i + 1 comes in and slice i - 1 goes out while slice i is computed.  Only for problems
+  // the attention kernels would not split (a slice must give the same bits as the whole), without a cache of key
+  // norms (indexed by the whole problem's head count), and when the side streams exist.
+  int slices = 1;
+  const size_t q_bytes = (size_t)p->batch * p->n_q_heads * head_bytes;
+  if (!p->k_inv_norm && attn_parts_bound(p) == 1 && q_bytes >= ((size_t)8 << 20)) {
+    if (p->n_kv_heads % 4 == 0) slices = 4;
+    else if (p->n_kv_heads % 2 == 0) slices = 2;
   }
-  st = quoka_prefill_chunk(p, q_dev, k_cache, v_cache, out_dev, nullptr, nullptr, ws, ws_bytes, stream);
-  if (st != QUOKA_OK) return st;
-  QUOKA_TRY_CUDA(cudaMemcpyAsync(out_host, out_dev, q_bytes, cudaMemcpyDeviceToHost, cs));
+  HostPipe* hp = slices > 1 ? host_pipe_for_current_device() : nullptr;
+  if (!hp) {
+    QUOKA_TRY_CUDA(copy_in(0, p->n_kv_heads, cs));
+    st = quoka_prefill_chunk(p, q_dev, k_cache, v_cache, out_dev, nullptr, nullptr, ws, ws_bytes, stream);
+    if (st != QUOKA_OK) return st;
+    QUOKA_TRY_CUDA(copy_out(0, p->n_kv_heads, cs));
+    return QUOKA_OK;
+  }
+  const int kv_per = p->n_kv_heads / slices;
+  quoka_params sub = *p;
+  sub.n_kv_heads = kv_per;
+  sub.n_q_heads = kv_per * G;
+  QUOKA_TRY_CUDA(cudaEventRecord(hp->fork, cs));
+  QUOKA_TRY_CUDA(cudaStreamWaitEvent(hp->h2d, hp->fork, 0));
+  for (int i = 0; i < slices; ++i) {
+    const int kv0 = i * kv_per;
+    QUOKA_TRY_CUDA(copy_in(kv0, kv_per, hp->h2d));
+    QUOKA_TRY_CUDA(cudaEventRecord(hp->in[i], hp->h2d));
+    QUOKA_TRY_CUDA(cudaStreamWaitEvent(cs, hp->in[i], 0));
+    st = prefill_chunk_impl(&sub, static_cast<char*>(q_dev) + (size_t)kv0 * G * head_bytes,
+                            static_cast<char*>(k_cache) + (size_t)kv0 * p->kv_stride_h * es,
+                            static_cast<char*>(v_cache) + (size_t)kv0 * p->kv_stride_h * es,
+                            static_cast<char*>(out_dev) + (size_t)kv0 * G * head_bytes, nullptr, nullptr, ws, ws_bytes,
+                            stream, /*with_split=*/false);
+    if (st != QUOKA_OK) return st;
+    QUOKA_TRY_CUDA(cudaEventRecord(hp->done[i], cs));
+    QUOKA_TRY_CUDA(cudaStreamWaitEvent(hp->d2h, hp->done[i], 0));
+    QUOKA_TRY_CUDA(copy_out(kv0, kv_per, hp->d2h));
+  }
+  QUOKA_TRY_CUDA(cudaEventRecord(hp->join, hp->d2h));
+  QUOKA_TRY_CUDA(cudaStreamWaitEvent(cs, hp->join, 0));
   return QUOKA_OK;
 }
 

@@ -243,18 +243,25 @@ def test_runs_are_bit_identical(impl):
             assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
 
 
-def test_host_buffer_entry_point_matches_device_entry_point():
-    gp = problem(11, n_q=8, n_kv=2, T=2000, C=256, n_retain=32, kv_budget=256)
+@pytest.mark.parametrize("shape", [dict(n_q=8, n_kv=2, T=2000, C=256, n_retain=32, kv_budget=256),
+                                   # large enough to be cut into four slices of KV groups that overlap their copies
+                                   dict(n_q=32, n_kv=8, T=3000, C=2048, n_retain=64, kv_budget=700),
+                                   dict(batch=2, n_q=12, n_kv=6, T=[1500, 800], C=1536, n_retain=64, kv_budget=300)],
+                         ids=["small", "four-slices", "two-slices-batch-2"])
+def test_host_buffer_entry_point_matches_device_entry_point(shape):
+    gp = problem(11, **shape)
     api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
     torch.cuda.synchronize()
     want = gp.out.clone()
-    T, C = 2000, 256
+    C = shape["C"]
+    Ts = [int(t) for t in gp.inp.ctx_len]
     q_host = gp.inp.q.contiguous().pin_memory()
-    k_new = gp.inp.k[:, :, T:T + C].contiguous().pin_memory()
-    v_new = gp.inp.v[:, :, T:T + C].contiguous().pin_memory()
+    k_new = torch.stack([gp.inp.k[s, :, T:T + C] for s, T in enumerate(Ts)]).contiguous().pin_memory()
+    v_new = torch.stack([gp.inp.v[s, :, T:T + C] for s, T in enumerate(Ts)]).contiguous().pin_memory()
     out_host = torch.zeros_like(q_host).pin_memory()
-    gp.k[:, :, T:T + C].zero_()
-    gp.v[:, :, T:T + C].zero_()
+    for s, T in enumerate(Ts):
+        gp.k[s, :, T:T + C].zero_()
+        gp.v[s, :, T:T + C].zero_()
     q_dev = torch.zeros_like(gp.q)
     gp.out.zero_()
     ctx_host = gp.inp.ctx_len.clone()
