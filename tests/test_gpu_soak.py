@@ -1,13 +1,15 @@
 """A seeded sweep of irregular shapes through the whole path: every stage of the staged calls against the oracle
 (chain validation, all attention rows), then the fused call bit for bit against the staged calls.  The shapes mix
 batch sizes, GQA ratios, head dims, dtypes, chunk lengths on and off the 128-row tiles, empty / one-row / long caches,
-key budgets as counts and as fractions, contiguous and paged caches."""
+key budgets as counts and as fractions, contiguous and paged caches.  The dense chunk attention of the same problem
+(the speed-up denominator; with a long cache and few heads it runs split into parts) is checked on one sequence."""
 import numpy as np
 import pytest
 import torch
 
 from paper_2602_08722_b200 import api, synth
-from tests.parity import GpuProblem, check_chain
+from oracle import quoka_oracle as O
+from tests.parity import GpuProblem, check_attention, check_chain, f64
 
 pytestmark = pytest.mark.gpu
 
@@ -31,7 +33,7 @@ def shape(seed):
                 kv_budget=kv_budget, frac=frac, paged=paged)
 
 
-@pytest.mark.parametrize("seed", list(range(9000, 9024)))
+@pytest.mark.parametrize("seed", list(range(9000, 9036)))
 def test_random_shape(seed):
     c = shape(seed)
     inp = synth.make_chunk_inputs(seed, c["batch"], c["n_q"], c["n_kv"], c["d"], c["T"] if c["batch"] > 1 else c["T"][0],
@@ -49,4 +51,12 @@ def test_random_shape(seed):
         torch.cuda.synchronize()
         assert torch.equal(idx2, staged_idx) and torch.equal(cnt2, staged_cnt), c
         assert torch.equal(gp.out, staged_out), c
+    s_chk = seed % c["batch"]
+    gp.out.zero_()
+    api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+    torch.cuda.synchronize()
+    q, k, v, T = gp.oracle_inputs(s_chk)
+    want, lse = O.dense_chunk_attention(q, k, v, T)
+    check_attention(f64(gp.out[s_chk]), want, c["dtype"])
+    assert np.abs(f64(gp.lse[s_chk]) - lse).max() <= 2e-3, c
     assert api.quoka_last_device_status(gp.ws) == 0
