@@ -270,6 +270,45 @@ def test_host_buffer_entry_point_matches_device_entry_point(shape):
     assert torch.equal(out_host, want.cpu())
 
 
+def test_host_buffer_entry_point_replayed_from_a_cuda_graph():
+    # the sliced call forks to the library's two copy streams and joins again: captured as one graph and replayed
+    shape = dict(n_q=32, n_kv=8, T=3000, C=2048, n_retain=64, kv_budget=700)
+    gp = problem(12, **shape)
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, None, None, gp.ws)
+    torch.cuda.synchronize()
+    want = gp.out.clone()
+    T, C = shape["T"], shape["C"]
+    q_host = gp.inp.q.contiguous().pin_memory()
+    k_new = gp.inp.k[:, :, T:T + C].contiguous().pin_memory()
+    v_new = gp.inp.v[:, :, T:T + C].contiguous().pin_memory()
+    out_host = torch.zeros_like(q_host).pin_memory()
+    q_dev = torch.zeros_like(gp.q)
+    ctx_host = gp.inp.ctx_len.clone()
+
+    def run():
+        api.quoka_prefill_chunk_host(gp.p, ctx_host, q_host, k_new, v_new, out_host, q_dev, gp.k, gp.v, gp.out, gp.ws)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run()                      # first use makes the copy streams: before any capture
+        side.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            run()
+    torch.cuda.synchronize()
+    for _ in range(2):
+        out_host.zero_()
+        gp.out.zero_()
+        q_dev.zero_()
+        gp.k[:, :, T:T + C].zero_()
+        gp.v[:, :, T:T + C].zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out_host, want.cpu())
+    assert api.quoka_last_device_status(gp.ws) == 0
+
+
 # ---------------------------------------------------------------- selection step alone: exact integer parity
 @pytest.mark.parametrize("T,B", [(5000, 600), (1024, 1), (1025, 1024), (33, 7), (70000, 8400)])
 def test_select_keys_exact_with_planted_ties(T, B):
