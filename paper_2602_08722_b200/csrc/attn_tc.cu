@@ -113,116 +113,14 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
       tc_fence_after();
       const int lim = visible_cols(tile_rows<SPARSE>(g, t), row);
       const bool masked = !__all_sync(0xFFFFFFFFu, lim >= kKeyTile);
-      // ---- pass 1: the row maximum.  All four 32-column loads are issued together (one tensor-memory round
-      // trip).  The first 96 scores stay in registers for pass 2, the last 32 are read once more there (under the
-      // third block's exponentials): all 128 alive next to a block of exponentials in flight do not fit the 168
-      // registers, and 96 fit only because P is stored 16 columns at a time and the rare rescale below works in
-      // 8-column pieces.
-      float mx;
-      uint32_t v0[96];                                         // the first 96 scores stay in registers for pass 2
-      {
-        uint32_t c3[32];
-        tmem_ld32(s_addr, v0);
-        tmem_ld32(s_addr + 32, v0 + 32);
-        tmem_ld32(s_addr + 64, v0 + 64);
-        tmem_ld32(s_addr + 96, c3);
-        tmem_wait_ld();
-        uint32_t (&a0)[32] = *reinterpret_cast<uint32_t (*)[32]>(v0);
-        uint32_t (&a1)[32] = *reinterpret_cast<uint32_t (*)[32]>(v0 + 32);
-        uint32_t (&a2)[32] = *reinterpret_cast<uint32_t (*)[32]>(v0 + 64);
-        mx = fmaxf(fmaxf(max32(a0, masked, 0, lim), max32(a1, masked, 32, lim)),
-                   fmaxf(max32(a2, masked, 64, lim), max32(c3, masked, 96, lim)));
-      }
-      const float m_tile = mx * scale_log2;
-      // ---- lazy rescale of the accumulator: only when some row's maximum grew by more than the threshold
-      const bool grow = m_tile > m_run + kRescaleThreshold;
-      if (__any_sync(0xFFFFFFFFu, grow)) {
-        const float m_new = fmaxf(m_run, m_tile);
-        if (t > skip_x) {
-          const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
-          l_run *= alpha;
-#pragma unroll 1
-          for (int c = 0; c < D / 8; ++c) {                       // rare: small pieces, few registers
-            uint32_t r[8];
-            tmem_ld8(o_addr + c * 8, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-            tmem_st8(o_addr + c * 8, r);
-          }
-          tmem_wait_st();
-        }
-        m_run = m_new;
-      }
-      const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-      // ---- pass 2: p = 2^(s*scale - m) in four blocks of 32 keys.  bf16 P goes over the first 64 columns of S
-      // (block b of P lands on columns 16b..16b+15, all of them read already) and each half of the tile is handed to
-      // the MMA issuer as soon as it is stored, so the first PV products run under the second half's arithmetic.
-      const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m_use, -m_use);
-      uint64_t psa[2] = {0ull, 0ull};                           // four running sums as two packed pairs
-      uint32_t vb[32];
-#pragma unroll
-      for (int blk = 0; blk < 4; ++blk) {
-        if (blk == 2) tmem_ld32(s_addr + 96, vb);              // under the third block's exponentials
-        if (blk == 3) {
-          tmem_wait_ld();
-          if (masked) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) if (96 + i >= lim) vb[i] = 0xFF800000u;   // -inf: exp2 gives exactly 0
-          }
-        }
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint32_t e0 = blk < 3 ? v0[blk * 32 + 2 * i] : vb[2 * i], e1 = blk < 3 ? v0[blk * 32 + 2 * i + 1] : vb[2 * i + 1];
-          float x0, x1;
-          unpack2(fma2(pack2u(e0, e1), sc2, nm2), x0, x1);
-          const float p0 = ex2(x0), p1 = ex2(x1);
-          psa[i & 1] = add2(psa[i & 1], pack2(p0, p1));
-          const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-          pk[i] = *reinterpret_cast<const uint32_t*>(&b2);
-        }
-        tmem_st16(s_addr + blk * 16, pk);
-        if (blk & 1) {
-          tmem_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&p_full[2 * x + (blk >> 1)]);
-        }
-      }
-      float ps0, ps1, ps2, ps3;
-      unpack2(psa[0], ps0, ps1);
-      unpack2(psa[1], ps2, ps3);
-      l_run += (ps0 + ps1) + (ps2 + ps3);
+      attn_softmax_tile<D>(s_addr, o_addr, lim, masked, scale_log2, t == skip_x, lane, m_run, l_run,
+                           [&](int half) { mbar_arrive(&p_full[2 * x + half]); });
     }
     // ---- epilogue: O / l -> bf16 -> global
     if constexpr (!SPLIT) {
       if (ok && active_x && mbar_wait(&o_full[x], 0, wc)) {
         tc_fence_after();
-        const float inv = 1.f / l_run;
-        const bool store = row < P.chunk;
-        __nv_bfloat16* orow = out + (long long)s * P.o_sb + (long long)h * P.o_sh + (long long)row * P.o_st;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(o_addr + c * 32, r);
-          tmem_wait_ld();
-          if (store) {
-#pragma unroll
-            for (int v4 = 0; v4 < 4; ++v4) {
-              uint32_t w[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
-                                                                 __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
-                w[i] = *reinterpret_cast<const uint32_t*>(&b2);
-              }
-              *reinterpret_cast<uint4*>(orow + c * 32 + v4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          }
-        }
-        if (store && lse)
-          lse[((long long)s * P.n_q + h) * P.chunk + row] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+        attn_store_row<D>(P, o_addr, m_run, l_run, s, h, row, out, lse);
       }
     } else {
       const bool have = ok && active_x && mbar_wait(&o_full[x], 0, wc);
