@@ -357,22 +357,13 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
 // Split attention.  A grid of fewer CTAs than half the SMs (short chunks, few heads) leaves most of the GPU idle
 // while every CTA walks its whole key sequence; cutting each row block's tiles into parts fills it.  A part costs a
 // start-up and a pass over the partial results, so parts keep at least six tiles.
-static int attn_sm_count() {
-  static int n = []() {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return v;
-  }();
-  return n;
-}
 static long long attn_jobs(const quoka_params* p) {
   return (long long)p->n_q_heads * ((p->chunk_len + 2 * kQTile - 1) / (2 * kQTile)) * p->batch;
 }
 int attn_split_parts(const quoka_params* p, int tiles) {
   if (p->dtype != QUOKA_BF16) return 1;
   const long long jobs = attn_jobs(p);
-  long long parts = attn_sm_count() / jobs;
+  long long parts = device_sm_count() / jobs;
   if (parts > tiles / 6) parts = tiles / 6;
   if (parts > 8) parts = 8;
   return parts < 1 ? 1 : (int)parts;

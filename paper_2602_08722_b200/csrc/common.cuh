@@ -154,6 +154,7 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 
 // Launch with optional thread-block cluster width and, if `chained`, programmatic stream serialisation.
 void log_launch(const char* kernel, dim3 grid, dim3 block, size_t smem, int cluster, bool chained);
+int device_sm_count();
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(const char* name, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,

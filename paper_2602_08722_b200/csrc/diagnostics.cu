@@ -40,6 +40,17 @@ __global__ void __launch_bounds__(32) wait_timeout_selftest_kernel(int32_t* stat
   if (threadIdx.x == 0) *gave_up = ok ? 0 : 1;
 }
 
+// SMs of the current device (looked up once per process).
+int device_sm_count() {
+  static int n = []() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return v;
+  }();
+  return n;
+}
+
 }  // namespace quoka
 
 using namespace quoka;

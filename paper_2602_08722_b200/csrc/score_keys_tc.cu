@@ -388,16 +388,6 @@ bool encode_kv_tensor_map(CUtensorMap* out, const quoka_params* p, const void* c
   return encode_tensor_map_bf16(out, cache, 4, dims, strides, box);
 }
 
-static int sm_count() {
-  static int n = []() {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return v;
-  }();
-  return n;
-}
-
 bool score_keys_tc_supported(const quoka_params* p) {
   if (p->dtype != QUOKA_BF16) return false;
   const int N = p->n_retain < p->chunk_len ? p->n_retain : p->chunk_len;
@@ -421,7 +411,7 @@ quoka_status launch_score_keys_tc(const quoka_params* p, const DevParams& P, con
   if (!encode_kv_tensor_map(&tm_k, p, k, 64)) return QUOKA_ERR_CUDA;
   ScoreArgs A{N, pl.n_pad, pl.n_parts, pl.box_rows, pl.q_rows, pl.stages, chained ? 1 : 0};
   const long long max_tiles = (long long)P.batch * P.n_kv * ((P.max_ctx + kTileKeys - 1) / kTileKeys);
-  int grid = sm_count();
+  int grid = device_sm_count();
   if (grid <= 0) return QUOKA_ERR_CUDA;
   if (max_tiles < grid) grid = (int)max_tiles;
   if (grid <= 0) return QUOKA_OK;
