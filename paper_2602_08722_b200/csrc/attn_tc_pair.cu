@@ -6,9 +6,11 @@
 // 256 rows of S (or O), 128 per CTA, with the K (or V) operand split between the two CTAs' shared memories.
 //   S = Q K^T : each CTA supplies its own Q tile and 64 of the tile's 128 keys (all 128 elements of each).
 //   O += P V  : each CTA supplies its own P (tensor memory) and 64 of V's 128 columns (all 128 keys).
-// So a CTA fetches HALF of every K and V tile, and per key tile and Q tile the tensor core reads 48 KB + 16 KB of
-// a CTA's shared memory instead of 64 KB + 32 KB.  The one-CTA kernel is co-limited by the shared-memory port
-// (256 KB per step at 128 B / clock = 2048 clocks, exactly the time of its products); here a step moves 160 KB.
+// So a CTA fetches HALF of every K and V tile (the 16-byte cp.async gather of listed rows tops out near 20 bytes per
+// clock and SM, which a one-CTA step of 64 KB all but needs), its loaders execute half the instructions, and per
+// key tile and Q tile the tensor core reads 48 KB + 16 KB of a CTA's shared memory instead of 64 KB + 32 KB.  A
+// step's time itself is set by one Q tile's chain S ready -> softmax -> P ready -> PV -> next QK^T and changes little:
+// measured against the one-CTA kernel, 1 % (listed rows) to 4 % (whole tiles, paged serving mix) faster.
 //
 // Roles per CTA as in the one-CTA kernel (8 softmax warps, 3 loader warps, warp 11), except:
 //   * only the first CTA's warp 11 issues MMAs.  A slot of its ring is ready when its own loaders AND the second
