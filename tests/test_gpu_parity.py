@@ -604,3 +604,21 @@ def test_split_attention_in_the_one_cta_kernel(d, n_q, n_kv):
         check_attention(f64(gp.out[s]), want, "bf16")
         assert np.abs(f64(gp.lse[s]) - lse).max() <= 2e-3
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+@pytest.mark.gpu
+def test_f32_rows_that_one_key_dominates_keep_the_thousands_of_small_weights():
+    """A shape from a randomised soak: f32, 5000 listed rows, and chunk rows whose softmax puts 0.99 on one key.
+    Summed one by one in fp32, the other 5000 weights (each below half an ulp of the running sum) vanished, 5e-5 of
+    the denominator and 2.6e-4 of an output of size 3.1; the scalar kernel's sums are compensated since."""
+    inp = synth.make_chunk_inputs(20062, 2, 4, 2, 64, [9000, 63], 200, "f32")
+    gp = GpuProblem(inp, 1, 5000, 0.0)
+    gp.run_staged()
+    check_chain(gp)
+    s = 0
+    q, k, v, T = gp.oracle_inputs(s)
+    cnt = int(gp.k_cnt[s])
+    idx = gp.k_idx[s].cpu().numpy()[:, :cnt]
+    want, lse = O.sparse_attention(q, k, v, T, [idx[kv] for kv in range(idx.shape[0])])
+    assert np.abs(f64(gp.out[s]) - want).max() <= 2e-5       # ten times inside the f32 tolerance
+    assert np.abs(f64(gp.lse[s]) - lse).max() <= 1e-5
