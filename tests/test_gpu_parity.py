@@ -622,3 +622,36 @@ def test_f32_rows_that_one_key_dominates_keep_the_thousands_of_small_weights():
     want, lse = O.sparse_attention(q, k, v, T, [idx[kv] for kv in range(idx.shape[0])])
     assert np.abs(f64(gp.out[s]) - want).max() <= 2e-5       # ten times inside the f32 tolerance
     assert np.abs(f64(gp.lse[s]) - lse).max() <= 1e-5
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n_q,n_kv,d,T,C,frac,paged,fac", [
+    (8, 2, 128, 4100, 300, 0.9, False, 6.0),       # CTA pairs, split into parts
+    (4, 4, 128, 3000, 257, 0.5, True, 8.0),        # one-CTA kernel (one query head per KV head), paged
+    (8, 2, 64, 2500, 200, 0.9, False, 6.0),        # head_dim 64
+    (32, 8, 128, 3000, 512, 0.3, False, 5.0)])     # two row blocks per head, unsplit
+def test_logits_far_beyond_the_lazy_rescale_threshold(n_q, n_kv, d, T, C, frac, paged, fac):
+    """The tensor-core kernels move the reference point of their exponentials (and rescale the accumulator in
+    tensor memory) only when a row's maximum outgrows it by 2^32.  Unit-variance inputs never get there, so here
+    the queries are scaled up and the keys grow along the cache: one row's logits span several hundred powers of
+    two and the maximum climbs from tile to tile, which also gives the parts of a split launch reference points
+    hundreds of powers of two apart."""
+    inp = synth.make_chunk_inputs(705, 1, n_q, n_kv, d, T, C, "bf16")
+    inp.q = (inp.q.float() * fac).to(torch.bfloat16)
+    ramp = torch.linspace(0.5, fac, inp.k.shape[2]).view(1, 1, -1, 1)
+    inp.k = (inp.k.float() * ramp).to(torch.bfloat16)
+    if paged:
+        inp = synth.to_paged(inp, 5)
+    gp = GpuProblem(inp, 16, 0, frac, paged=paged)
+    q, k, v, Ts = gp.oracle_inputs(0)
+    span = (q[0, -1] @ k[0, :Ts + C].T) / np.sqrt(d) * 1.4427
+    assert span.max() - span.min() > 300           # powers of two, far beyond the threshold of 32
+    gp.run_staged()
+    check_chain(gp)
+    gp.out.zero_()
+    api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+    torch.cuda.synchronize()
+    want, lse = O.dense_chunk_attention(q, k, v, Ts)
+    check_attention(f64(gp.out[0]), want, "bf16")
+    assert np.abs(f64(gp.lse[0]) - lse).max() <= 2e-3 * max(1.0, np.abs(lse).max() / 50)
+    assert api.quoka_last_device_status(gp.ws) == 0
