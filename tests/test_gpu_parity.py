@@ -655,3 +655,33 @@ def test_logits_far_beyond_the_lazy_rescale_threshold(n_q, n_kv, d, T, C, frac, 
     check_attention(f64(gp.out[0]), want, "bf16")
     assert np.abs(f64(gp.lse[0]) - lse).max() <= 2e-3 * max(1.0, np.abs(lse).max() / 50)
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+def _equal_queries(inp): inp.q[:] = inp.q[:, :, :1]
+def _equal_keys(inp): inp.k[:, :, :2000] = inp.k[:, :, :1]
+def _zero_keys(inp): inp.k[:, :, 100:900] = 0
+def _zero_queries(inp): inp.q[:, 0] = 0
+def _zero_values(inp): inp.v[:] = 0
+def _tiny_keys(inp): inp.k[:, :, :2000] = inp.k[:, :, :2000] * 1e-3
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("mutate", [_equal_queries, _equal_keys, _zero_keys, _zero_queries, _zero_values, _tiny_keys],
+                         ids=lambda f: f.__name__.strip("_"))
+def test_degenerate_inputs(mutate, dtype):
+    """Inputs on which the method's quantities tie or vanish: every query of a head equal (all cosines to the mean
+    query tie: ranks by position), every cached key equal (all scores tie: lowest positions first), keys and queries
+    of norm zero (the eps of the normalisation decides), values all zero, keys a thousand times smaller than queries."""
+    inp = synth.make_chunk_inputs(800, 1, 8, 2, 128, 2000, 300, dtype)
+    mutate(inp)
+    gp = GpuProblem(inp, 16, 300, 0.0)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged)
+    assert torch.isfinite(gp.out.float()).all()
+    assert api.quoka_last_device_status(gp.ws) == 0
