@@ -685,3 +685,39 @@ def test_degenerate_inputs(mutate, dtype):
     assert torch.equal(gp.out, staged)
     assert torch.isfinite(gp.out.float()).all()
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+def _token_major(t):            # (b, heads, rows, d) view of a (b, rows, heads, d) buffer
+    return t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+
+
+def _padded_rows(t, pad):       # rows `pad` elements longer than head_dim
+    big = torch.zeros(*t.shape[:3], t.shape[3] + pad, dtype=t.dtype, device=t.device)
+    big[..., : t.shape[3]] = t
+    return big[..., : t.shape[3]]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("layout", ["token-major", "padded"])
+@pytest.mark.parametrize("n_q,n_kv,d,T,C,frac", [(8, 2, 128, [4100, 700], 129, 0.9), (4, 4, 64, 1500, 200, 0.3),
+                                                 (32, 8, 128, 2000, 512, 0.12)])
+def test_strided_layouts(n_q, n_kv, d, T, C, frac, layout, dtype):
+    """q, out and the KV cache are described by element strides: the same problem with queries and cache stored
+    token-major ((b, rows, heads, d), the layout projections usually write) and with padded rows."""
+    batch = len(T) if isinstance(T, list) else 1
+    inp = synth.make_chunk_inputs(900, batch, n_q, n_kv, d, T, C, dtype)
+    gp = GpuProblem(inp, 16, 0, frac)
+    fq, fk = (_token_major, _token_major) if layout == "token-major" else (lambda t: _padded_rows(t, 64), lambda t: _padded_rows(t, 8))
+    gp.q, gp.out = fq(gp.q), fq(torch.zeros_like(gp.q))
+    gp.k, gp.v = fk(gp.k), fk(gp.v)
+    assert not gp.q.is_contiguous() and not gp.k.is_contiguous()
+    gp.p = api.make_params(gp.q, gp.k, gp.out, gp.ctx_len, n_retain=16, kv_budget=0, budget_frac=frac, max_ctx_len=gp.max_ctx)
+    gp.run_staged()
+    check_chain(gp)
+    staged = gp.out.clone()
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged)
+    assert api.quoka_last_device_status(gp.ws) == 0
