@@ -721,3 +721,33 @@ def test_strided_layouts(n_q, n_kv, d, T, C, frac, layout, dtype):
     torch.cuda.synchronize()
     assert torch.equal(gp.out, staged)
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("n_q,n_kv,d,T,C", [(8, 2, 128, 3000, 300), (4, 4, 64, 1500, 200), (8, 2, 128, 4100, 1)])
+@pytest.mark.parametrize("scale", [0.03, 0.3])
+def test_softmax_scale_given_by_the_caller(scale, n_q, n_kv, d, T, C, dtype):
+    """softmax_scale != 0 replaces 1 / sqrt(head_dim) in Eq. 1 / Eq. 2 (every attention kernel: CTA pairs, one CTA,
+    scalar, and the one-query kernel), and does not touch the selection."""
+    inp = synth.make_chunk_inputs(950, 1, n_q, n_kv, d, T, C, dtype)
+    gp = GpuProblem(inp, 16, 0, 0.5)
+    gp.p.softmax_scale = scale
+    gp.run_staged()
+    q, k, v, Ts = gp.oracle_inputs(0)
+    cnt = int(gp.k_cnt[0])
+    idx = gp.k_idx[0].cpu().numpy()[:, :cnt]
+    want, lse = O.sparse_attention(q, k, v, Ts, [idx[kv] for kv in range(n_kv)], scale=scale)
+    check_attention(f64(gp.out[0]), want, dtype)
+    assert np.abs(f64(gp.lse[0]) - lse).max() <= 2e-3
+    sel_scaled = gp.k_idx.clone()
+    gp.p.softmax_scale = 0.0
+    gp.run_staged()
+    assert torch.equal(gp.k_idx, sel_scaled)
+    gp.p.softmax_scale = scale
+    gp.out.zero_()
+    api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+    torch.cuda.synchronize()
+    want, lse = O.dense_chunk_attention(q, k, v, Ts, scale=scale)
+    check_attention(f64(gp.out[0]), want, dtype)
+    assert np.abs(f64(gp.lse[0]) - lse).max() <= 2e-3
