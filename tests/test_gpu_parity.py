@@ -69,6 +69,14 @@ def test_gqa_ratios(G, impl):
     check_chain(gp)
 
 
+@pytest.mark.parametrize("n_q,n_kv", [(12, 2), (10, 5), (14, 7), (9, 3), (5, 5)])
+def test_gqa_ratios_that_are_not_powers_of_two(n_q, n_kv):
+    # 6 and 2 query heads per KV head run as CTA pairs (with 5 or 7 KV heads), 3 and 1 in the one-CTA kernel
+    gp = problem(960, batch=2, n_q=n_q, n_kv=n_kv, T=[4100, 200], C=129, n_retain=16, kv_budget=0, budget_frac=0.9)
+    gp.run_staged()
+    check_chain(gp)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("paged", [False, True])
 def test_batched_variable_lengths(paged, impl):
