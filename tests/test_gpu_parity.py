@@ -759,3 +759,18 @@ def test_softmax_scale_given_by_the_caller(scale, n_q, n_kv, d, T, C, dtype):
     want, lse = O.dense_chunk_attention(q, k, v, Ts, scale=scale)
     check_attention(f64(gp.out[0]), want, dtype)
     assert np.abs(f64(gp.lse[0]) - lse).max() <= 2e-3
+
+
+@pytest.mark.gpu
+def test_split_attention_over_a_200k_row_cache():
+    # 8 heads x 1 row block = 8 CTAs before the split, 782 list tiles: eight parts of ~100 tiles each
+    inp = synth.make_chunk_inputs(970, 1, 8, 2, 128, 200000, 256, "bf16")
+    gp = GpuProblem(inp, 32, 0, 0.5)
+    gp.run_staged()
+    check_chain(gp, attn_rows=48)
+    staged = gp.out.clone()
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged)
+    assert api.quoka_last_device_status(gp.ws) == 0
