@@ -119,7 +119,7 @@ quoka_status quoka_kv_budget_cap(const quoka_params* p, int32_t* cap);
  * The first 256 bytes hold the device status word, which the caller sets to zero
  * once after allocating; the rest is scratch whose contents mean nothing between
  * calls.  Two calls that share a workspace must not overlap on the GPU.
- * For problems whose attention grid is far smaller than the GPU (few heads, a short
+ * For problems whose attention grid is smaller than the GPU (few heads, a short
  * chunk) the size includes room for the partial results of the split attention
  * kernel (each row block's keys are cut into up to 8 parts, one CTA each, and added
  * up in part order: results are reproducible from run to run, and differ from the

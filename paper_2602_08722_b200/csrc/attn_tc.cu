@@ -354,19 +354,29 @@ attn_tc_kernel(DevParams P, const __grid_constant__ CUtensorMap tm_q, const __gr
 }
 
 // ---------------------------------------------------------------------------------------------- host
-// Split attention.  A grid of fewer CTAs than half the SMs (short chunks, few heads) leaves most of the GPU idle
-// while every CTA walks its whole key sequence; cutting each row block's tiles into parts fills it.  A part costs a
-// start-up and a pass over the partial results, so parts keep at least six tiles.
+// Split attention.  A grid of fewer CTAs than SMs (short chunks, few heads) leaves part of the GPU idle while
+// every CTA walks its whole key sequence; cutting each row block's tiles into parts, one CTA each, fills it.
+// The number of parts minimises  waves(parts) * (tiles / parts + 6):  a part costs about six tiles' time of
+// start-up, partial results and merge (the model fits the measured times of 1 to 5 parts on grids of 32 to 288 CTAs
+// within 3 %), parts keep at least six tiles, and a split has to promise 3 % to be taken.  Grids of a wave or more
+// stay whole: their sparse jobs are too short to gain, and the partial results of long dense ones would take
+// hundreds of megabytes.
 static long long attn_jobs(const quoka_params* p) {
   return (long long)p->n_q_heads * ((p->chunk_len + 2 * kQTile - 1) / (2 * kQTile)) * p->batch;
 }
 int attn_split_parts(const quoka_params* p, int tiles) {
   if (p->dtype != QUOKA_BF16) return 1;
-  const long long jobs = attn_jobs(p);
-  long long parts = device_sm_count() / jobs;
-  if (parts > tiles / 6) parts = tiles / 6;
-  if (parts > 8) parts = 8;
-  return parts < 1 ? 1 : (int)parts;
+  const long long jobs = attn_jobs(p), sms = device_sm_count();
+  if (sms <= 0 || jobs >= sms) return 1;
+  const double t = tiles + (p->chunk_len + 2 * kQTile - 1) / (2 * kQTile);   // plus the chunk's own tiles, on average
+  int best = 1;
+  double best_cost = t;
+  for (int parts = 2; parts <= 8 && parts <= tiles / 6; ++parts) {
+    const long long waves = (jobs * parts + sms - 1) / sms;
+    const double cost = (double)waves * (t / parts + 6.0);
+    if (cost < 0.97 * best_cost) { best = parts; best_cost = cost; }
+  }
+  return best;
 }
 size_t attn_split_partial_bytes(const quoka_params* p, int parts) {
   return parts <= 1 ? 0 : (size_t)attn_jobs(p) * parts * 2 * kSplitTileFloats * sizeof(float);

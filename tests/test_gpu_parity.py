@@ -774,3 +774,26 @@ def test_split_attention_over_a_200k_row_cache():
     torch.cuda.synchronize()
     assert torch.equal(gp.out, staged)
     assert api.quoka_last_device_status(gp.ws) == 0
+
+
+@pytest.mark.gpu
+def test_split_attention_of_a_grid_between_half_a_wave_and_a_wave():
+    # 8 heads x 10 row blocks = 80 CTAs of ~130 tiles: three parts each (two waves of a third beat one wave of a whole)
+    inp = synth.make_chunk_inputs(971, 1, 8, 2, 128, 17000, 2560, "bf16")
+    gp = GpuProblem(inp, 64, 0, 0.9)
+    gp.run_staged()
+    check_chain(gp, attn_rows=64)
+    staged = gp.out.clone()
+    gp.out.zero_()
+    api.quoka_prefill_chunk(gp.p, gp.q, gp.k, gp.v, gp.out, gp.k_idx, gp.k_cnt, gp.ws)
+    torch.cuda.synchronize()
+    assert torch.equal(gp.out, staged)
+    gp.out.zero_()
+    api.quoka_dense_chunk_attn(gp.p, gp.q, gp.k, gp.v, gp.out, gp.lse, gp.ws)
+    torch.cuda.synchronize()
+    q, k, v, Ts = gp.oracle_inputs(0)
+    heads, rows = stratified_rows(8, 2560, 48, 3)
+    idx_all = [np.arange(Ts)] * 2
+    want = O.sparse_attention_rows(q, k, v, Ts, idx_all, heads, rows)       # every cached row listed = Eq. 2
+    check_attention(f64(gp.out[0])[heads, rows], want, "bf16")
+    assert api.quoka_last_device_status(gp.ws) == 0
